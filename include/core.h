@@ -1,0 +1,172 @@
+/*
+ * core.h -- C ABI of the B200 (sm_100a) CORE library.
+ *
+ * CORE (Common Random Reconstruction) compresses a d-dimensional vector to m
+ * scalars by projecting it on m common Gaussian vectors and rebuilds an
+ * unbiased estimate from the scalars by regenerating the same vectors
+ * (Algorithm 1 of the paper).  With n machines the estimate of the mean
+ * gradient is  gtilde = 1/(n m) sum_i sum_j <g_i, xi_j> xi_j  (Section 4,
+ * definition of the estimator used by Algorithm 2).
+ *
+ * Common random vectors (the paper asks only for "a common random number
+ * generator"; this is the generator this library fixes):
+ *   words   Philox4x32-10, key = (seed mod 2^32, seed >> 32),
+ *           counter = (q mod 2^32, q >> 32, j, t); q = k >> 2 is the block of
+ *           four coordinates, j the 0-based vector index, t the round.
+ *   uniform u(w) = ((w >> 9) + 1/2) 2^-23.
+ *   normal  Box-Muller on (w0,w1) and (w2,w3): r = sqrt(-2 ln u(w_even)),
+ *           theta = 2 pi u(w_odd); xi_j[4q..4q+3] = (r_a cos th_a, r_a sin th_a,
+ *           r_b cos th_b, r_b sin th_b).
+ * The vectors are never stored: every kernel regenerates what it needs.
+ *
+ * Conventions for every entry point
+ *   - Pointers named *_dev are DEVICE pointers owned by the caller; *_host are
+ *     HOST pointers owned by the caller.  The context owns only its workspace.
+ *   - Work is enqueued on the context's stream (core_set_stream; default: the
+ *     legacy default stream) and the call returns without synchronising,
+ *     except the *_host entry points, which return after their last copy has
+ *     completed, and any call that has to grow the workspace (cudaMalloc).
+ *   - Return value: CORE_OK or a negative error code.  A failing call launches
+ *     nothing for CORE_EINVAL; outputs are unspecified after any error, but no
+ *     call writes outside the extents stated here.  Nothing prints or aborts.
+ *   - One context may be used by one host thread at a time.
+ */
+#ifndef CORE_B200_CORE_H
+#define CORE_B200_CORE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct core_ctx core_ctx;
+typedef struct core_ls core_ls;
+
+enum {
+    CORE_OK = 0,
+    CORE_EINVAL = -1, /* null pointer, non-positive size, ld < d, unknown dtype */
+    CORE_ENOMEM = -2, /* workspace allocation failed */
+    CORE_ECUDA = -3   /* CUDA runtime error; code via core_last_cuda_error */
+};
+
+enum { CORE_F32 = 0, CORE_BF16 = 1 };
+
+/* ---- context ------------------------------------------------------------- */
+
+/*
+ * Create a context for vectors of dimension d >= 1 compressed to m >= 1 scalars
+ * with the common generator keyed by seed.  Round counter starts at t = 0.
+ * The ten Philox round keys are derived here, once.  Binds to the CUDA device
+ * current at the time of the call.
+ */
+int core_init(core_ctx **out, uint64_t seed, int64_t d, int32_t m);
+int core_destroy(core_ctx *ctx);
+
+/* cuda_stream is a cudaStream_t passed as an opaque pointer (NULL: default stream). */
+int core_set_stream(core_ctx *ctx, void *cuda_stream);
+
+/*
+ * Round index t selects which "fresh" set xi_1..xi_m is generated (Algorithm 1,
+ * first step; Algorithm 2, first step of the loop).  Projection and
+ * reconstruction of one communication round must use the same t.
+ */
+int core_set_round(core_ctx *ctx, uint32_t t);
+uint32_t core_get_round(const core_ctx *ctx);
+
+/* Bytes of device workspace the context currently holds. */
+size_t core_workspace_bytes(const core_ctx *ctx);
+
+const char *core_strerror(int code);
+int core_last_cuda_error(const core_ctx *ctx);
+
+/* ---- the round ------------------------------------------------------------- */
+
+/*
+ * Projection: P[i*m + j] = <g_i, xi_j>, i < n, j < m (Algorithm 1, sender's
+ * step; Algorithm 2, "machine i sends p_ij").
+ *   G_dev   n rows of d elements, row i at element offset i*ldg (ldg >= d),
+ *           dtype CORE_F32 (float) or CORE_BF16 (bfloat16, widened exactly).
+ *           Rows whose byte address and stride are multiples of 16 take the
+ *           asynchronous-copy path; any other alignment is handled by an
+ *           element-wise path with the same result.
+ *   P_dev   n*m floats, row-major.
+ * fp32 multiply-add with two-level fp32 accumulation and a fixed reduction
+ * order: results are bitwise reproducible for a given (n, m, d, dtype).
+ * n > 16 is processed in groups of 16 machines.  May grow the workspace.
+ */
+int core_project(core_ctx *ctx, const void *G_dev, int dtype, int32_t n, int64_t ldg, float *P_dev);
+
+/*
+ * Aggregation at the central machine (Algorithm 2, "the central machine sends
+ * the combined p_ij back"), in the mean convention of the Section-4 estimator
+ * (prefactor 1/(n m)):  pbar[j] = (1/n) sum_i P[i*m + j], i ascending.
+ */
+int core_aggregate(core_ctx *ctx, const float *P_dev, int32_t n, float *pbar_dev);
+
+/*
+ * Reconstruction: gtilde[k] = (1/m) sum_j pbar[j] xi_j[k], k < d (Algorithm 1,
+ * receiver's step; the equation following Algorithm 1).  gtilde_dev: d floats,
+ * each written exactly once.
+ */
+int core_reconstruct(core_ctx *ctx, const float *pbar_dev, float *gtilde_dev);
+
+/*
+ * One whole communication round (Algorithm 2, steps 1-4): project, aggregate,
+ * reconstruct with the current t, then t <- t + 1.  pbar_dev (m floats) receives
+ * the aggregated message; gtilde_dev (d floats) the estimate.
+ */
+int core_round(core_ctx *ctx, const void *G_dev, int dtype, int32_t n, int64_t ldg, float *pbar_dev,
+               float *gtilde_dev);
+
+/*
+ * The same round with HOST buffers: G_host (n rows, stride ldg elements) is
+ * streamed to the device in coordinate slabs that are projected as they
+ * arrive; gtilde_host (d floats) and pbar_host (m floats) are copied back, the
+ * reconstruction being produced and copied slab by slab.  Pinned host memory
+ * gives asynchronous copies; pageable memory works but serialises.  Returns
+ * after the last copy has completed.  t <- t + 1.
+ */
+int core_round_host(core_ctx *ctx, const void *G_host, int dtype, int32_t n, int64_t ldg,
+                    float *pbar_host, float *gtilde_host);
+
+/* ---- least-squares CORE-GD driver (Algorithm 2) ----------------------------- */
+
+/*
+ * f(x) = (1/n) sum_i 1/(2 rows) ||A_i x - b_i||^2 : the ridge-separable form of
+ * Section 4 with quadratic loss and no ridge term.  A_dev is n x rows x d floats
+ * row-major, b_dev n x rows floats; both are borrowed (must outlive the handle).
+ * The handle owns the gradient matrix G[n x d] and its partial sums.
+ */
+int core_ls_create(core_ls **out, const float *A_dev, const float *b_dev, int32_t n, int32_t rows,
+                   int64_t d);
+int core_ls_destroy(core_ls *ls);
+
+/*
+ * One iteration of Algorithm 2: g_i = A_i^T (A_i x - b_i) / rows for every
+ * machine, one round with the context's current t (then t <- t + 1), and
+ * x <- x - h * gtilde.  x_dev: d floats, updated in place.  ctx must have been
+ * created with the same d.
+ */
+int core_gd_step(core_ctx *ctx, core_ls *ls, float h, float *x_dev);
+
+/* loss_dev[0] = f(x) as a double, computed on the device. */
+int core_ls_loss(core_ctx *ctx, core_ls *ls, const float *x_dev, double *loss_dev);
+
+/* G_out_dev[i*d + k] = g_i[k] at x (the machine gradients alone; n*d floats). */
+int core_ls_gradients(core_ctx *ctx, core_ls *ls, const float *x_dev, float *G_out_dev);
+
+/* ---- generator windows (for checking the generator itself) ------------------- */
+
+/* words_dev[4*(q-q0) + l] = word l of block q of vector j, q0 <= q < q0+nq, current t. */
+int core_debug_philox(core_ctx *ctx, uint32_t j, uint64_t q0, int64_t nq, uint32_t *words_dev);
+/* z_dev[4*(q-q0) + l] = xi_j[4q + l]. */
+int core_debug_gaussians(core_ctx *ctx, uint32_t j, uint64_t q0, int64_t nq, float *z_dev);
+/* Box-Muller alone: z_dev[4b..4b+3] from the caller's words_dev[4b..4b+3], b < nb. */
+int core_debug_box_muller(core_ctx *ctx, const uint32_t *words_dev, int64_t nb, float *z_dev);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

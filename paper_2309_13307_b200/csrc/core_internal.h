@@ -1,0 +1,72 @@
+// Internal declarations shared by the translation units of the CORE library.
+#pragma once
+
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "core_rng.cuh"
+
+namespace core {
+
+constexpr int kThreads = 256;        // threads per CTA in the round kernels
+constexpr int kMaxGroup = 16;        // machines handled by one projection pass
+
+// Launch geometry of one projection pass, fixed by (n, m, d, dtype) on the host.
+struct ProjectPlan {
+    int nb;           // machines per pass rounded up to 1, 2, 4, 8 or 16
+    int jt;           // vectors per thread
+    int uq;           // coordinate blocks per thread per step
+    int tile_q;       // coordinate blocks (of 4) per shared-memory tile
+    int tj;           // threads across vectors (power of two)
+    int tq;           // threads across coordinate blocks = kThreads / tj
+    int grid_x;       // CTAs across coordinates
+    int grid_y;       // CTAs across vectors
+    int64_t tiles;    // ceil(d / (4 * tile_q))
+    size_t smem;      // dynamic shared memory per CTA
+};
+
+ProjectPlan make_project_plan(int32_t n_group, int32_t m, int64_t d, int dtype, int sm_count);
+
+// One projection pass over coordinates [0, d) of rows G + i*ldg, i < n <= 16.
+// q_base is the global index of the block holding coordinate 0 of G (non-zero when G
+// is a slab of a longer vector).  Writes partial[(c * n + i) * m + j], c < plan.grid_x.
+cudaError_t launch_project(const ProjectPlan &plan, const RoundKeys &keys, uint32_t t, const void *G,
+                           int dtype, int32_t n, int64_t ldg, int64_t d, int32_t m, uint64_t q_base,
+                           float *partial, cudaStream_t stream);
+
+// P[i*m+j] = (accumulate ? P[i*m+j] : 0) + sum_c partial[c][i][j], c ascending.
+cudaError_t launch_finish_project(const float *partial, int chunks, int32_t n, int32_t m, float *P,
+                                  bool accumulate, cudaStream_t stream);
+
+cudaError_t launch_aggregate(const float *P, int32_t n, int32_t m, float *pbar, cudaStream_t stream);
+
+// out[k - k_begin] = gtilde[k] for k in [k_begin, k_end); k_begin must be a multiple of 2048.
+cudaError_t launch_reconstruct(const RoundKeys &keys, uint32_t t, const float *pbar, int32_t m,
+                               int64_t k_begin, int64_t k_end, float *out, int sm_count,
+                               cudaStream_t stream);
+
+// x[k] -= h * g[k]
+cudaError_t launch_axpy(float *x, const float *g, float h, int64_t d, cudaStream_t stream);
+
+cudaError_t launch_debug_philox(const RoundKeys &keys, uint32_t t, uint32_t j, uint64_t q0, int64_t nq,
+                                uint32_t *words, cudaStream_t stream);
+cudaError_t launch_debug_gaussians(const RoundKeys &keys, uint32_t t, uint32_t j, uint64_t q0, int64_t nq,
+                                   float *z, cudaStream_t stream);
+cudaError_t launch_debug_box_muller(const uint32_t *words, int64_t nb, float *z, cudaStream_t stream);
+
+// Least squares: each machine's rows are split over ctas_per_machine CTAs; every CTA
+// leaves a partial gradient and a partial sum of squared residuals.
+struct LsPlan {
+    int ctas_per_machine;
+    int rows_per_cta;
+};
+LsPlan make_ls_plan(int32_t n, int32_t rows, int64_t d, int sm_count);
+cudaError_t launch_ls_partial(const LsPlan &plan, const float *A, const float *b, const float *x, int32_t n,
+                              int32_t rows, int64_t d, float *part, double *res2, cudaStream_t stream);
+cudaError_t launch_ls_reduce(const LsPlan &plan, const float *part, int32_t n, int32_t rows, int64_t d,
+                             float *G, cudaStream_t stream);
+cudaError_t launch_ls_loss(const LsPlan &plan, const double *res2, int32_t n, int32_t rows, double *loss,
+                           cudaStream_t stream);
+
+}  // namespace core

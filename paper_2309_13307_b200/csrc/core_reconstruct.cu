@@ -1,0 +1,207 @@
+// Fused regenerate-and-reconstruct kernel: gtilde[k] = (1/m) sum_j pbar[j] xi_j[k]
+// (Algorithm 1, receiver's step; the equation that follows Algorithm 1).
+//
+// A thread owns UQ coordinate blocks of four coordinates and runs over all vectors j,
+// regenerating xi_j for its blocks from the same counters the projection used.  The
+// part of the Philox evaluation that depends only on the block is computed once per
+// thread; the part that depends only on j is tabulated per CTA in shared memory next
+// to pbar[j], so the loop reads one 16-byte broadcast per j.  Every output coordinate
+// is written exactly once, as a 16-byte store where alignment allows.
+#include "core_internal.h"
+
+namespace core {
+
+namespace {
+
+constexpr int kRecUQ = 2;                         // coordinate blocks per thread per group
+constexpr int kGroupQ = kThreads * kRecUQ;        // blocks per CTA step
+constexpr int kJChunk = 2048;                     // vectors tabulated at a time (32 KB)
+
+struct ReconstructArgs {
+    const float *pbar;
+    float *out;
+    int64_t k_begin;
+    int64_t k_end;
+    int m;
+    int vec_ok;       // out + 4*(q - q_begin) is 16-byte aligned
+    uint32_t t;
+    RoundKeys keys;
+};
+
+__global__ void __launch_bounds__(kThreads, 2)
+reconstruct_kernel(const __grid_constant__ ReconstructArgs a) {
+    __shared__ uint4 table[kJChunk];              // {JPart.x0, JPart.x2, JPart.w3, bits of pbar[j]}
+    const int tid = threadIdx.x;
+    const uint64_t q_begin = (uint64_t)a.k_begin >> 2;
+    const uint64_t q_end = ((uint64_t)a.k_end + 3) >> 2;
+    const uint64_t groups = (q_end - q_begin + kGroupQ - 1) / kGroupQ;
+    const float inv_m = 1.0f / (float)a.m;
+
+    bool have_table = false;
+    uint32_t table_qhi = 0;
+
+    for (uint64_t grp = blockIdx.x; grp < groups; grp += gridDim.x) {
+        // q_begin is a multiple of kGroupQ (launch_reconstruct checks), so a group never
+        // straddles a multiple of 2^32 and all its blocks share the high counter word.
+        const uint64_t gq0 = q_begin + grp * kGroupQ;
+        const uint32_t grp_qhi = (uint32_t)(gq0 >> 32);
+
+        float4 acc[kRecUQ];
+        QPart qp[kRecUQ];
+        uint64_t qv[kRecUQ];
+#pragma unroll
+        for (int u = 0; u < kRecUQ; ++u) {
+            qv[u] = gq0 + (uint64_t)(tid + u * kThreads);
+            qp[u] = philox_qpart((uint32_t)qv[u], a.t, a.keys);
+            acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+
+        for (int j0 = 0; j0 < a.m; j0 += kJChunk) {
+            const int jn = min(kJChunk, a.m - j0);
+            const bool rebuild = !have_table || table_qhi != grp_qhi || a.m > kJChunk;
+            if (rebuild) {
+                __syncthreads();                  // everyone is done with the previous table
+                for (int jj = tid; jj < jn; jj += kThreads) {
+                    const JPart jp = philox_jpart((uint32_t)(j0 + jj), grp_qhi, a.keys);
+                    table[jj] = make_uint4(jp.x0, jp.x2, jp.w3, __float_as_uint(a.pbar[j0 + jj]));
+                }
+                __syncthreads();
+                have_table = true;
+                table_qhi = grp_qhi;
+            }
+#pragma unroll 2
+            for (int jj = 0; jj < jn; ++jj) {
+                const uint4 e = table[jj];
+                const float p = __uint_as_float(e.w);
+#pragma unroll
+                for (int u = 0; u < kRecUQ; ++u) {
+                    JPart jp;
+                    jp.x0 = e.x;
+                    jp.x2 = e.y;
+                    jp.w3 = e.z;
+                    const float4 z = box_muller4(philox_combine(jp, qp[u], a.keys));
+                    acc[u].x = fmaf(p, z.x, acc[u].x);
+                    acc[u].y = fmaf(p, z.y, acc[u].y);
+                    acc[u].z = fmaf(p, z.z, acc[u].z);
+                    acc[u].w = fmaf(p, z.w, acc[u].w);
+                }
+            }
+        }
+
+#pragma unroll
+        for (int u = 0; u < kRecUQ; ++u) {
+            if (qv[u] >= q_end) continue;
+            const float4 r = make_float4(acc[u].x * inv_m, acc[u].y * inv_m, acc[u].z * inv_m, acc[u].w * inv_m);
+            const int64_t off = (int64_t)((qv[u] - q_begin) << 2);        // offset into out
+            const int64_t k = (int64_t)(qv[u] << 2);
+            if (a.vec_ok && k + 4 <= a.k_end) {
+                *reinterpret_cast<float4 *>(a.out + off) = r;
+            } else {
+                const float vals[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                for (int l = 0; l < 4; ++l)
+                    if (k + l < a.k_end) a.out[off + l] = vals[l];
+            }
+        }
+    }
+}
+
+__global__ void axpy_kernel(float *__restrict__ x, const float *__restrict__ g, float h, int64_t d) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < d; k += stride)
+        x[k] = fmaf(-h, g[k], x[k]);
+}
+
+struct DebugArgs {
+    uint64_t q0;
+    int64_t nq;
+    uint32_t j;
+    uint32_t t;
+    RoundKeys keys;
+};
+
+__global__ void debug_philox_kernel(const __grid_constant__ DebugArgs a, uint4 *words) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; r < a.nq; r += stride) {
+        const uint64_t q = a.q0 + (uint64_t)r;
+        words[r] = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), a.j, a.t, a.keys);
+    }
+}
+
+// Goes through the split evaluation the round kernels use, so that path is what is checked.
+__global__ void debug_gaussians_kernel(const __grid_constant__ DebugArgs a, float4 *z) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; r < a.nq; r += stride) {
+        const uint64_t q = a.q0 + (uint64_t)r;
+        const JPart jp = philox_jpart(a.j, (uint32_t)(q >> 32), a.keys);
+        const QPart qp = philox_qpart((uint32_t)q, a.t, a.keys);
+        z[r] = box_muller4(philox_combine(jp, qp, a.keys));
+    }
+}
+
+__global__ void debug_box_muller_kernel(const uint4 *__restrict__ words, int64_t nb, float4 *z) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; r < nb; r += stride)
+        z[r] = box_muller4(words[r]);
+}
+
+unsigned grid_for(int64_t items, int threads, int cap) {
+    int64_t g = (items + threads - 1) / threads;
+    if (g < 1) g = 1;
+    if (g > cap) g = cap;
+    return (unsigned)g;
+}
+
+}  // namespace
+
+cudaError_t launch_reconstruct(const RoundKeys &keys, uint32_t t, const float *pbar, int32_t m,
+                               int64_t k_begin, int64_t k_end, float *out, int sm_count,
+                               cudaStream_t stream) {
+    if (k_end <= k_begin) return cudaSuccess;
+    if (k_begin % (4 * kGroupQ) != 0) return cudaErrorInvalidValue;
+    ReconstructArgs a{};
+    a.pbar = pbar;
+    a.out = out;
+    a.k_begin = k_begin;
+    a.k_end = k_end;
+    a.m = m;
+    a.vec_ok = (reinterpret_cast<uintptr_t>(out) % 16) == 0 ? 1 : 0;
+    a.t = t;
+    a.keys = keys;
+    const int64_t nq = ((k_end + 3) >> 2) - (k_begin >> 2);
+    const int64_t groups = (nq + kGroupQ - 1) / kGroupQ;
+    int64_t grid = (int64_t)sm_count * 2;
+    if (grid > groups) grid = groups;
+    reconstruct_kernel<<<(unsigned)grid, kThreads, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_axpy(float *x, const float *g, float h, int64_t d, cudaStream_t stream) {
+    axpy_kernel<<<grid_for(d, 256, 148 * 8), 256, 0, stream>>>(x, g, h, d);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_debug_philox(const RoundKeys &keys, uint32_t t, uint32_t j, uint64_t q0, int64_t nq,
+                                uint32_t *words, cudaStream_t stream) {
+    if (nq <= 0) return cudaSuccess;
+    DebugArgs a{q0, nq, j, t, keys};
+    debug_philox_kernel<<<grid_for(nq, 256, 148 * 8), 256, 0, stream>>>(a, reinterpret_cast<uint4 *>(words));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_debug_gaussians(const RoundKeys &keys, uint32_t t, uint32_t j, uint64_t q0, int64_t nq,
+                                   float *z, cudaStream_t stream) {
+    if (nq <= 0) return cudaSuccess;
+    DebugArgs a{q0, nq, j, t, keys};
+    debug_gaussians_kernel<<<grid_for(nq, 256, 148 * 8), 256, 0, stream>>>(a, reinterpret_cast<float4 *>(z));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_debug_box_muller(const uint32_t *words, int64_t nb, float *z, cudaStream_t stream) {
+    if (nb <= 0) return cudaSuccess;
+    debug_box_muller_kernel<<<grid_for(nb, 256, 148 * 8), 256, 0, stream>>>(
+        reinterpret_cast<const uint4 *>(words), nb, reinterpret_cast<float4 *>(z));
+    return cudaGetLastError();
+}
+
+}  // namespace core
