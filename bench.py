@@ -1,0 +1,344 @@
+#!/usr/bin/env python
+"""Benchmark of the CORE round on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one pass of the whole path over the projection-dimension sweep workload:
+d = 1e9 fp32 coordinates, n = 2 machines, and for every m in {8, 64, 512, 4096} one round
+(project -> aggregate -> reconstruct).  The metric counts coordinate x vector pairs: a step
+processes d * sum(m) of them per kernel.  The path does not shard (all machines are simulated
+on one GPU, no collectives), so N > 1 runs N independent replicas, one per GPU.
+
+Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "CORE round throughput (coords x m projected+reconstructed/s)"
+UNIT = "coord*vector pairs/s"
+SEED_DATA, SEED_XI = 0, 1
+SM_COUNT, LANES_PER_SM = 148, 128
+# Algorithmic lane-operations per generated Gaussian: Philox4x32-10 = (20 wide multiplies +
+# 20 three-input xors) / 4 words = 10; Box-Muller per pair = 2 x (shift, or, add) to form the
+# uniforms' floats ... counted as 12 per pair = 6 per Gaussian.  Plus one FMA per machine
+# (project) or one FMA (reconstruct).
+OPS_PER_GAUSSIAN = 16
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--d", type=int, default=None, help="override the coordinate count (development)")
+    ap.add_argument("--m", type=int, nargs="*", default=None, help="override the m sweep (development)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    return ap.parse_args()
+
+
+# ---- clocks ---------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---- CPU oracle leg -----------------------------------------------------------------------
+
+def oracle_mini_round(d_s: int, m_s: int, n_s: int, threads: int):
+    """One whole oracle round on a bounded sample; returns (seconds, units)."""
+    import math
+    from concurrent.futures import ThreadPoolExecutor
+
+    import numpy as np
+
+    import core_inputs
+    import oracle
+
+    G = core_inputs.gradients(n_s, d_s, seed=SEED_DATA).numpy()
+    oracle.lib()
+    piece = max(4, (d_s // threads + 3) // 4 * 4)
+    cuts = list(range(0, d_s, piece)) + [d_s]
+    spans = list(zip(cuts[:-1], cuts[1:]))
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        def proj(span):
+            return [[oracle.project_slice(SEED_XI, 0, j, G[i], span[0], span[1]) for j in range(m_s)]
+                    for i in range(n_s)]
+        parts = list(ex.map(proj, spans))
+        P = np.array([[math.fsum(p[i][j] for p in parts) for j in range(m_s)] for i in range(n_s)])
+        pbar = oracle.aggregate(P)
+        list(ex.map(lambda span: oracle.reconstruct_slice(SEED_XI, 0, pbar, span[0], span[1]), spans))
+    dt = time.perf_counter() - t0
+    return dt, d_s * m_s
+
+
+def cpu_baseline_sample(budget_s: float = 15.0):
+    threads = max(1, min(os.cpu_count() or 1, 64))
+    n_s, m_s = 2, 8
+    d_s = 1 << 18
+    dt, units = oracle_mini_round(d_s, m_s, n_s, threads)          # calibration
+    scale = max(1, min(64, int(budget_s / max(dt, 1e-3))))
+    if scale > 1:
+        d_s *= scale
+        dt, units = oracle_mini_round(d_s, m_s, n_s, threads)
+    return {"value": units / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"one whole oracle round (project+aggregate+reconstruct, fp64) at d={d_s}, m={m_s}, "
+                      f"n={n_s}, N(0,1) gradients, coordinate range split over {threads} host threads; "
+                      f"{dt:.1f} s"}
+
+
+def run_reference(args):
+    """The reference arm of this build is the CPU oracle, as it stands, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    threads = max(1, min(os.cpu_count() or 1, 64))
+    n_s, m_s, d_s = 2, 8, 1 << 24
+    for _ in range(args.warmup):
+        oracle_mini_round(1 << 16, m_s, n_s, threads)
+    total_t, total_u = 0.0, 0
+    for _ in range(args.steps):
+        dt, units = oracle_mini_round(d_s, m_s, n_s, threads)
+        total_t += dt
+        total_u += units
+    value = total_u / total_t
+    sample = (f"each step: one whole oracle round at d={d_s}, m={m_s}, n={n_s} (a bounded sample of the "
+              f"d=1e9 sweep workload), split over {threads} host threads")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "sweep: d=1e9 fp32, n=2, m in {8,64,512,4096} (bounded sample per step)"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+# ---- GPU leg ---------------------------------------------------------------------------------
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import core_inputs
+    import paper_2309_13307_b200 as core_mod
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    core_mod.lib()                                   # fails loudly if the CUDA library is missing
+    w = core_inputs.WORKLOADS["sweep"]
+    d = args.d or w.d
+    ms = tuple(args.m) if args.m else w.m
+    n = w.n
+    G = core_inputs.gradients(n, d, seed=SEED_DATA + rank, dist=w.dist, dtype=w.dtype, device="cuda")
+    ctxs = {m: core_mod.Core(SEED_XI, d, m) for m in ms}
+    P = {m: torch.empty((n, m), dtype=torch.float32, device="cuda") for m in ms}
+    pbar = {m: torch.empty(m, dtype=torch.float32, device="cuda") for m in ms}
+    gt = torch.empty(d, dtype=torch.float32, device="cuda")
+    units_per_step = d * sum(ms)
+
+    def ev():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record()
+        return e
+
+    marks = []                                        # (m, e0, e_proj, e_agg, e_rec) per timed round
+
+    def step(timed: bool):
+        for m in ms:
+            c = ctxs[m]
+            e0 = ev() if timed else None
+            c.core_project(G, P[m])
+            e1 = ev() if timed else None
+            c.core_aggregate(P[m], pbar[m])
+            e2 = ev() if timed else None
+            c.core_reconstruct(pbar[m], gt)
+            e3 = ev() if timed else None
+            c.core_set_round(c.core_get_round() + 1)
+            if timed:
+                marks.append((m, e0, e1, e2, e3))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step(False)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(args.steps):
+        step(True)
+    stop.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    elapsed_ms = start.elapsed_time(stop)
+    if world > 1:
+        tmax = torch.tensor([elapsed_ms], device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(tmax.item())
+    value = world * units_per_step * args.steps / (elapsed_ms * 1e-3)
+
+    # per-kernel times (averages over the timed launches)
+    per_m = {}
+    for m in ms:
+        rows = [r for r in marks if r[0] == m]
+        tp = statistics.mean(r[1].elapsed_time(r[2]) for r in rows)
+        tr = statistics.mean(r[3].elapsed_time(r[4]) for r in rows)
+        ta = statistics.mean(r[2].elapsed_time(r[3]) for r in rows)
+        per_m[m] = (tp, ta, tr)
+
+    # end to end through the host-buffer entry point
+    e2e = None
+    if not args.no_e2e:
+        Gh = torch.empty((n, d), dtype=G.dtype).pin_memory()
+        Gh.copy_(G)
+        gt_h = torch.empty(d, dtype=torch.float32).pin_memory()
+        pbar_h = {m: torch.empty(m, dtype=torch.float32).pin_memory() for m in ms}
+        for m in ms:                                   # warm-up: allocates the slabs
+            if m == min(ms):
+                ctxs[m].core_round_host(Gh, pbar_h[m], gt_h)
+        barrier()
+        e2e_steps = 1
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            for m in ms:
+                ctxs[m].core_round_host(Gh, pbar_h[m], gt_h)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        if world > 1:
+            tt = torch.tensor([dt], device="cuda")
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            dt = float(tt.item())
+        e2e = {"value": world * units_per_step * e2e_steps / dt, "unit": UNIT,
+               "h2d_bytes_per_step": len(ms) * n * d * G.element_size(),
+               "d2h_bytes_per_step": len(ms) * (d * 4) + sum(ms) * 4,
+               "steps": e2e_steps, "how": "core_round_host from pinned host buffers, host clock around the "
+                                          "blocking calls (each returns after its last copy)"}
+        del Gh, gt_h
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # roofline of the dominant kernel (largest share of the step)
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except OSError:
+        pass
+    sm_max = (clocks or {}).get("sm_max_mhz") or peaks.get("sm_max_mhz") or 1965.0
+    alu_peak = SM_COUNT * LANES_PER_SM * sm_max * 1e6          # lane-operations per second
+    kernels = []
+    for m in ms:
+        tp, ta, tr = per_m[m]
+        kernels.append(("project", m, tp, OPS_PER_GAUSSIAN + n, n * d * G.element_size()))
+        kernels.append(("reconstruct", m, tr, OPS_PER_GAUSSIAN + 1, 4 * d))
+    name, m_dom, t_dom, ops_per_unit, hbm_bytes = max(kernels, key=lambda k: k[2])
+    achieved = d * m_dom * ops_per_unit / (t_dom * 1e-3)
+    roofline = {"bound": "alu", "kernel": f"{name} m={m_dom}", "achieved": achieved / 1e12, "peak": alu_peak / 1e12,
+                "unit": "Tlane-op/s", "frac": achieved / alu_peak, "traffic": None,
+                "ops_per_unit": ops_per_unit, "ms_per_launch": t_dom,
+                "peak_source": f"148 SM x 128 fp32/int32 lanes x {sm_max:.0f} MHz (max SM clock)",
+                "hbm_frac_of_measured": (hbm_bytes / (t_dom * 1e-3)) / (peaks.get("hbm_gbs", 6650.0) * 1e9)}
+    sweep = []
+    for kname, m, t_ms, ops, hb in kernels:
+        sweep.append({"kernel": kname, "m": m, "ms": round(t_ms, 4), "units_per_s": d * m / (t_ms * 1e-3),
+                      "alu_frac": d * m * ops / (t_ms * 1e-3) / alu_peak,
+                      "hbm_frac": hb / (t_ms * 1e-3) / (peaks.get("hbm_gbs", 6650.0) * 1e9)})
+
+    cpu = None if args.no_cpu else cpu_baseline_sample()
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"sweep: d={d} fp32, n={n}, N(0,1) gradients, m in {list(ms)}; one round per m",
+                   "l2": "inputs (8 GB of gradients per replica) are larger than L2; no flush needed",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": 4 * len(ms) * args.steps,
+        "roofline": roofline, "sweep": sweep, "cpu_baseline": cpu,
+    }
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -166,6 +166,16 @@ int core_debug_gaussians(core_ctx *ctx, uint32_t j, uint64_t q0, int64_t nq, flo
 /* Box-Muller alone: z_dev[4b..4b+3] from the caller's words_dev[4b..4b+3], b < nb. */
 int core_debug_box_muller(core_ctx *ctx, const uint32_t *words_dev, int64_t nb, float *z_dev);
 
+/*
+ * Launch geometry the projection would use for n machines (one pass handles at most 16),
+ * m vectors and d coordinates on a device with sm_count SMs.  Host-only: touches no device.
+ * out[0..9] = machines per pass (rounded up to a power of two), vectors per thread,
+ * coordinate blocks per thread step, blocks per shared-memory tile, threads across
+ * vectors, threads across blocks, CTAs across coordinates, CTAs across vectors,
+ * tiles of d, dynamic shared memory bytes.
+ */
+int core_debug_project_plan(int32_t n, int32_t m, int64_t d, int dtype, int32_t sm_count, int64_t out[10]);
+
 #ifdef __cplusplus
 }
 #endif

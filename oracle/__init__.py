@@ -62,6 +62,10 @@ def lib() -> ctypes.CDLL:
             L.oracle_xi_block.restype = None
             L.oracle_xi_range.argtypes = [u64, u32, u32, i64, i64, vp]
             L.oracle_xi_range.restype = None
+            L.oracle_xi_words_many.argtypes = [u64, u32, u32, u64, i64, vp]
+            L.oracle_xi_words_many.restype = None
+            L.oracle_box_muller_many.argtypes = [vp, i64, vp]
+            L.oracle_box_muller_many.restype = None
             L.oracle_project_slice.argtypes = [u64, u32, u32, vp, ci, i64, i64]
             L.oracle_project_slice.restype = dbl
             L.oracle_project.argtypes = [u64, u32, i64, i32, i32, vp, ci, i64, vp]
@@ -131,9 +135,15 @@ def xi_words(seed: int, t: int, j: int, q: int) -> np.ndarray:
 def xi_words_range(seed: int, t: int, j: int, q0: int, q1: int) -> np.ndarray:
     """Raw words of blocks q0..q1-1 of vector j, shape [q1-q0, 4]."""
     out = np.zeros((q1 - q0, 4), dtype=np.uint32)
-    L = lib()
-    for r, q in enumerate(range(q0, q1)):
-        L.oracle_xi_words(seed, t, j, q, out[r].ctypes.data)
+    lib().oracle_xi_words_many(seed, t, j, q0, q1 - q0, _ptr(out))
+    return out
+
+
+def box_muller_many(words: np.ndarray) -> np.ndarray:
+    """Box-Muller of an [nb, 4] uint32 array of words; returns [nb, 4] float64."""
+    words = np.ascontiguousarray(words, dtype=np.uint32).reshape(-1, 4)
+    out = np.zeros(words.shape, dtype=np.float64)
+    lib().oracle_box_muller_many(_ptr(words), words.shape[0], _ptr(out))
     return out
 
 

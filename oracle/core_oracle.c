@@ -89,6 +89,15 @@ void oracle_xi_range(uint64_t seed, uint32_t t, uint32_t j, int64_t k0, int64_t 
     for (int64_t k = k0; k < k1; ++k) out[k - k0] = xi_at(seed, t, j, k);
 }
 
+/* convenience loops over the two functions above, for checking many blocks at once */
+void oracle_xi_words_many(uint64_t seed, uint32_t t, uint32_t j, uint64_t q0, int64_t nq, uint32_t *out) {
+    for (int64_t r = 0; r < nq; ++r) oracle_xi_words(seed, t, j, q0 + (uint64_t)r, out + 4 * r);
+}
+
+void oracle_box_muller_many(const uint32_t *w, int64_t nb, double *z) {
+    for (int64_t r = 0; r < nb; ++r) oracle_box_muller(w + 4 * r, z + 4 * r);
+}
+
 /* ---- gradient element access ---------------------------------------------- */
 
 /* dtype 0 float, 1 bfloat16 bit pattern (upper half of an fp32), 2 double. */

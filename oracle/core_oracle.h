@@ -58,6 +58,12 @@ void oracle_xi_block(uint64_t seed, uint32_t t, uint32_t j, uint64_t q, double z
 /* xi_j^{(t)}[k0 .. k1) written to out[0 .. k1-k0). */
 void oracle_xi_range(uint64_t seed, uint32_t t, uint32_t j, int64_t k0, int64_t k1, double *out);
 
+/* out[4r..4r+3] = words of block q0 + r, r < nq. */
+void oracle_xi_words_many(uint64_t seed, uint32_t t, uint32_t j, uint64_t q0, int64_t nq, uint32_t *out);
+
+/* z[4r..4r+3] = Box-Muller of w[4r..4r+3], r < nb. */
+void oracle_box_muller_many(const uint32_t *w, int64_t nb, double *z);
+
 /*
  * Projection (Algorithm 1, "M1 sends p_i = <a, xi_i>"; Algorithm 2, machine i
  * sends p_ij): sum over k in [k0,k1) of g[k] * xi_j[k], k ascending, fp64.

@@ -1,0 +1,274 @@
+"""ctypes binding of the CORE C ABI (``include/core.h``): argument marshalling only.
+
+Every function has the name of the C entry point it calls and takes torch tensors (device
+memory for ``*_dev`` arguments, host memory for ``*_host``).  Nothing is computed here, and
+there is no fallback: if ``libcore_b200.so`` cannot be loaded the import of a symbol raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+CORE_OK, CORE_EINVAL, CORE_ENOMEM, CORE_ECUDA = 0, -1, -2, -3
+CORE_F32, CORE_BF16 = 0, 1
+
+_lib = None
+
+_c = ctypes
+_SIGNATURES = {
+    "core_init": ([_c.POINTER(_c.c_void_p), _c.c_uint64, _c.c_int64, _c.c_int32], _c.c_int),
+    "core_destroy": ([_c.c_void_p], _c.c_int),
+    "core_set_stream": ([_c.c_void_p, _c.c_void_p], _c.c_int),
+    "core_set_round": ([_c.c_void_p, _c.c_uint32], _c.c_int),
+    "core_get_round": ([_c.c_void_p], _c.c_uint32),
+    "core_workspace_bytes": ([_c.c_void_p], _c.c_size_t),
+    "core_strerror": ([_c.c_int], _c.c_char_p),
+    "core_last_cuda_error": ([_c.c_void_p], _c.c_int),
+    "core_project": ([_c.c_void_p, _c.c_void_p, _c.c_int, _c.c_int32, _c.c_int64, _c.c_void_p], _c.c_int),
+    "core_aggregate": ([_c.c_void_p, _c.c_void_p, _c.c_int32, _c.c_void_p], _c.c_int),
+    "core_reconstruct": ([_c.c_void_p, _c.c_void_p, _c.c_void_p], _c.c_int),
+    "core_round": ([_c.c_void_p, _c.c_void_p, _c.c_int, _c.c_int32, _c.c_int64, _c.c_void_p, _c.c_void_p],
+                   _c.c_int),
+    "core_round_host": ([_c.c_void_p, _c.c_void_p, _c.c_int, _c.c_int32, _c.c_int64, _c.c_void_p,
+                         _c.c_void_p], _c.c_int),
+    "core_ls_create": ([_c.POINTER(_c.c_void_p), _c.c_void_p, _c.c_void_p, _c.c_int32, _c.c_int32, _c.c_int64],
+                       _c.c_int),
+    "core_ls_destroy": ([_c.c_void_p], _c.c_int),
+    "core_gd_step": ([_c.c_void_p, _c.c_void_p, _c.c_float, _c.c_void_p], _c.c_int),
+    "core_ls_loss": ([_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p], _c.c_int),
+    "core_ls_gradients": ([_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p], _c.c_int),
+    "core_debug_philox": ([_c.c_void_p, _c.c_uint32, _c.c_uint64, _c.c_int64, _c.c_void_p], _c.c_int),
+    "core_debug_gaussians": ([_c.c_void_p, _c.c_uint32, _c.c_uint64, _c.c_int64, _c.c_void_p], _c.c_int),
+    "core_debug_box_muller": ([_c.c_void_p, _c.c_void_p, _c.c_int64, _c.c_void_p], _c.c_int),
+    "core_debug_project_plan": ([_c.c_int32, _c.c_int32, _c.c_int64, _c.c_int, _c.c_int32,
+                                 _c.POINTER(_c.c_int64)], _c.c_int),
+}
+
+
+class CoreError(RuntimeError):
+    def __init__(self, code: int, where: str, cuda: int = 0):
+        self.code = code
+        self.cuda = cuda
+        msg = lib().core_strerror(code).decode()
+        super().__init__(f"{where}: {msg} (code {code}" + (f", CUDA error {cuda})" if cuda else ")"))
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library.  Raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if not os.path.exists(path):
+            raise RuntimeError(
+                f"{path} is missing: build it with `python -m paper_2309_13307_b200.build` "
+                "(needs nvcc); the CORE library has no non-CUDA path")
+        L = ctypes.CDLL(path)
+        for name, (argtypes, restype) in _SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.argtypes = argtypes
+            fn.restype = restype
+        _lib = L
+    return _lib
+
+
+def exported_symbols():
+    return list(_SIGNATURES)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return CORE_F32
+    if t.dtype == torch.bfloat16:
+        return CORE_BF16
+    raise TypeError(f"gradients must be float32 or bfloat16, not {t.dtype}")
+
+
+def _rows(G: torch.Tensor):
+    """(pointer, dtype code, n, ld) of a 2-D tensor whose rows are contiguous."""
+    if G.dim() != 2 or G.stride(1) != 1:
+        raise ValueError("G must be 2-D with unit stride along coordinates")
+    n = G.shape[0]
+    ld = G.stride(0) if n > 1 else max(G.stride(0), G.shape[1])
+    return G.data_ptr(), _dtype_code(G), n, ld
+
+
+def _dev(t: torch.Tensor, dtype, numel=None) -> int:
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"expected a contiguous CUDA tensor of {dtype}")
+    if numel is not None and t.numel() < numel:
+        raise ValueError(f"tensor too small: {t.numel()} < {numel}")
+    return t.data_ptr()
+
+
+def core_debug_project_plan(n: int, m: int, d: int, dtype: int = CORE_F32, sm_count: int = 148) -> dict:
+    out = (ctypes.c_int64 * 10)()
+    rc = lib().core_debug_project_plan(n, m, d, dtype, sm_count, out)
+    if rc != CORE_OK:
+        raise CoreError(rc, "core_debug_project_plan")
+    keys = ("nb", "jt", "uq", "tile_q", "tj", "tq", "grid_x", "grid_y", "tiles", "smem")
+    return dict(zip(keys, (int(v) for v in out)))
+
+
+class Core:
+    """A ``core_ctx``: fixed (seed, d, m), a round counter t, a stream and a workspace."""
+
+    def __init__(self, seed: int, d: int, m: int, stream: torch.cuda.Stream | None = None):
+        self._h = ctypes.c_void_p()
+        self.seed, self.d, self.m = int(seed), int(d), int(m)
+        rc = lib().core_init(ctypes.byref(self._h), self.seed, self.d, self.m)
+        if rc != CORE_OK:
+            self._h = ctypes.c_void_p()
+            raise CoreError(rc, "core_init")
+        self.core_set_stream(stream if stream is not None else torch.cuda.current_stream())
+
+    def _check(self, rc: int, where: str):
+        if rc != CORE_OK:
+            raise CoreError(rc, where, lib().core_last_cuda_error(self._h))
+
+    def close(self):
+        if getattr(self, "_h", None) and self._h.value:
+            lib().core_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- context ------------------------------------------------------------------
+    def core_set_stream(self, stream: torch.cuda.Stream):
+        self._check(lib().core_set_stream(self._h, ctypes.c_void_p(stream.cuda_stream)), "core_set_stream")
+
+    def core_set_round(self, t: int):
+        self._check(lib().core_set_round(self._h, int(t)), "core_set_round")
+
+    def core_get_round(self) -> int:
+        return int(lib().core_get_round(self._h))
+
+    def core_workspace_bytes(self) -> int:
+        return int(lib().core_workspace_bytes(self._h))
+
+    # -- the round ------------------------------------------------------------------
+    def core_project(self, G_dev: torch.Tensor, P_dev: torch.Tensor | None = None) -> torch.Tensor:
+        ptr, code, n, ld = _rows(G_dev)
+        if not G_dev.is_cuda or G_dev.shape[1] != self.d:
+            raise ValueError("G must be a CUDA tensor of shape [n, d]")
+        if P_dev is None:
+            P_dev = torch.empty((n, self.m), dtype=torch.float32, device=G_dev.device)
+        self._check(lib().core_project(self._h, ptr, code, n, ld, _dev(P_dev, torch.float32, n * self.m)),
+                    "core_project")
+        return P_dev
+
+    def core_aggregate(self, P_dev: torch.Tensor, pbar_dev: torch.Tensor | None = None) -> torch.Tensor:
+        n = P_dev.shape[0]
+        if pbar_dev is None:
+            pbar_dev = torch.empty(self.m, dtype=torch.float32, device=P_dev.device)
+        self._check(lib().core_aggregate(self._h, _dev(P_dev, torch.float32, n * self.m), n,
+                                         _dev(pbar_dev, torch.float32, self.m)), "core_aggregate")
+        return pbar_dev
+
+    def core_reconstruct(self, pbar_dev: torch.Tensor, gtilde_dev: torch.Tensor | None = None) -> torch.Tensor:
+        if gtilde_dev is None:
+            gtilde_dev = torch.empty(self.d, dtype=torch.float32, device=pbar_dev.device)
+        self._check(lib().core_reconstruct(self._h, _dev(pbar_dev, torch.float32, self.m),
+                                           _dev(gtilde_dev, torch.float32, self.d)), "core_reconstruct")
+        return gtilde_dev
+
+    def core_round(self, G_dev: torch.Tensor, pbar_dev: torch.Tensor | None = None,
+                   gtilde_dev: torch.Tensor | None = None):
+        ptr, code, n, ld = _rows(G_dev)
+        if not G_dev.is_cuda or G_dev.shape[1] != self.d:
+            raise ValueError("G must be a CUDA tensor of shape [n, d]")
+        if pbar_dev is None:
+            pbar_dev = torch.empty(self.m, dtype=torch.float32, device=G_dev.device)
+        if gtilde_dev is None:
+            gtilde_dev = torch.empty(self.d, dtype=torch.float32, device=G_dev.device)
+        self._check(lib().core_round(self._h, ptr, code, n, ld, _dev(pbar_dev, torch.float32, self.m),
+                                     _dev(gtilde_dev, torch.float32, self.d)), "core_round")
+        return pbar_dev, gtilde_dev
+
+    def core_round_host(self, G_host: torch.Tensor, pbar_host: torch.Tensor, gtilde_host: torch.Tensor):
+        ptr, code, n, ld = _rows(G_host)
+        if G_host.is_cuda or pbar_host.is_cuda or gtilde_host.is_cuda or G_host.shape[1] != self.d:
+            raise ValueError("core_round_host takes host tensors, G of shape [n, d]")
+        if pbar_host.dtype != torch.float32 or gtilde_host.dtype != torch.float32 or \
+                pbar_host.numel() < self.m or gtilde_host.numel() < self.d or \
+                not pbar_host.is_contiguous() or not gtilde_host.is_contiguous():
+            raise ValueError("pbar_host [m] and gtilde_host [d] must be contiguous float32")
+        self._check(lib().core_round_host(self._h, ptr, code, n, ld, pbar_host.data_ptr(),
+                                          gtilde_host.data_ptr()), "core_round_host")
+        return pbar_host, gtilde_host
+
+    # -- least squares ------------------------------------------------------------
+    def core_gd_step(self, ls: "LeastSquares", h: float, x_dev: torch.Tensor):
+        self._check(lib().core_gd_step(self._h, ls._h, float(h), _dev(x_dev, torch.float32, self.d)),
+                    "core_gd_step")
+        return x_dev
+
+    def core_ls_loss(self, ls: "LeastSquares", x_dev: torch.Tensor, loss_dev: torch.Tensor | None = None):
+        if loss_dev is None:
+            loss_dev = torch.empty(1, dtype=torch.float64, device=x_dev.device)
+        self._check(lib().core_ls_loss(self._h, ls._h, _dev(x_dev, torch.float32, self.d),
+                                       _dev(loss_dev, torch.float64, 1)), "core_ls_loss")
+        return loss_dev
+
+    def core_ls_gradients(self, ls: "LeastSquares", x_dev: torch.Tensor, G_out_dev: torch.Tensor | None = None):
+        if G_out_dev is None:
+            G_out_dev = torch.empty((ls.n, self.d), dtype=torch.float32, device=x_dev.device)
+        self._check(lib().core_ls_gradients(self._h, ls._h, _dev(x_dev, torch.float32, self.d),
+                                            _dev(G_out_dev, torch.float32, ls.n * self.d)), "core_ls_gradients")
+        return G_out_dev
+
+    # -- generator windows ----------------------------------------------------------
+    def core_debug_philox(self, j: int, q0: int, nq: int) -> torch.Tensor:
+        words = torch.empty((nq, 4), dtype=torch.int32, device="cuda")
+        self._check(lib().core_debug_philox(self._h, j, q0, nq, words.data_ptr()), "core_debug_philox")
+        return words
+
+    def core_debug_gaussians(self, j: int, q0: int, nq: int) -> torch.Tensor:
+        z = torch.empty((nq, 4), dtype=torch.float32, device="cuda")
+        self._check(lib().core_debug_gaussians(self._h, j, q0, nq, z.data_ptr()), "core_debug_gaussians")
+        return z
+
+    def core_debug_box_muller(self, words_dev: torch.Tensor) -> torch.Tensor:
+        nb = words_dev.numel() // 4
+        z = torch.empty((nb, 4), dtype=torch.float32, device=words_dev.device)
+        self._check(lib().core_debug_box_muller(self._h, _dev(words_dev, torch.int32, 4 * nb), nb, z.data_ptr()),
+                    "core_debug_box_muller")
+        return z
+
+
+class LeastSquares:
+    """A ``core_ls``: borrows A[n, rows, d] and b[n, rows] (kept alive here), owns the gradient scratch."""
+
+    def __init__(self, A_dev: torch.Tensor, b_dev: torch.Tensor):
+        if A_dev.dim() != 3 or b_dev.shape != A_dev.shape[:2]:
+            raise ValueError("A must be [n, rows, d] and b [n, rows]")
+        self.A, self.b = A_dev, b_dev
+        self.n, self.rows, self.d = (int(s) for s in A_dev.shape)
+        self._h = ctypes.c_void_p()
+        rc = lib().core_ls_create(ctypes.byref(self._h), _dev(A_dev, torch.float32), _dev(b_dev, torch.float32),
+                                  self.n, self.rows, self.d)
+        if rc != CORE_OK:
+            self._h = ctypes.c_void_p()
+            raise CoreError(rc, "core_ls_create")
+
+    def close(self):
+        if getattr(self, "_h", None) and self._h.value:
+            lib().core_ls_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

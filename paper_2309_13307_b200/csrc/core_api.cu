@@ -1,0 +1,451 @@
+// C ABI of the CORE library: argument checks, context, workspace and stream plumbing.
+// Every entry point is declared, with its contract, in include/core.h.
+#include "core.h"
+
+#include <new>
+
+#include "core_internal.h"
+
+using namespace core;
+
+struct core_ctx {
+    uint64_t seed;
+    int64_t d;
+    int32_t m;
+    uint32_t t;
+    int device;
+    int sm_count;
+    cudaStream_t stream;
+    RoundKeys keys;
+    void *ws;            // device workspace, grown on demand
+    size_t ws_bytes;
+    float *pbar;         // m floats, for callers that do not keep the message (gd step)
+    int last_cuda;
+    // host-streaming state (core_round_host), created on first use
+    cudaStream_t copy_stream, work_stream;
+    cudaEvent_t in_ready[2], in_free[2], out_ready[2], out_free[2];
+    bool host_ready;
+    void *slab;          // 2 input slabs + 2 output slabs
+    size_t slab_bytes;
+};
+
+struct core_ls {
+    const float *A;
+    const float *b;
+    int32_t n, rows;
+    int64_t d;
+    int device;
+    LsPlan plan;
+    float *res;          // n*rows
+    float *part;         // n*splits*d
+    float *G;            // n*d
+    float *gt;           // d
+};
+
+namespace {
+
+size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int cuda_fail(core_ctx *ctx, cudaError_t e) {
+    if (ctx) ctx->last_cuda = (int)e;
+    return e == cudaErrorMemoryAllocation ? CORE_ENOMEM : CORE_ECUDA;
+}
+
+#define CORE_CUDA(ctx, expr)                                  \
+    do {                                                      \
+        cudaError_t e__ = (expr);                             \
+        if (e__ != cudaSuccess) return cuda_fail((ctx), e__); \
+    } while (0)
+
+bool on_device(int device) {
+    int cur = -1;
+    return cudaGetDevice(&cur) == cudaSuccess && cur == device;
+}
+
+int ensure_workspace(core_ctx *ctx, size_t bytes) {
+    if (bytes <= ctx->ws_bytes) return CORE_OK;
+    if (ctx->ws) {
+        cudaError_t e = cudaFree(ctx->ws);   // waits for work that may still use it
+        ctx->ws = nullptr;
+        ctx->ws_bytes = 0;
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    }
+    bytes = round_up(bytes, (size_t)1 << 20);
+    cudaError_t e = cudaMalloc(&ctx->ws, bytes);
+    if (e != cudaSuccess) {
+        ctx->ws = nullptr;
+        cudaGetLastError();
+        ctx->last_cuda = (int)e;
+        return CORE_ENOMEM;
+    }
+    ctx->ws_bytes = bytes;
+    return CORE_OK;
+}
+
+bool valid_dtype(int dtype) { return dtype == CORE_F32 || dtype == CORE_BF16; }
+size_t elem_size(int dtype) { return dtype == CORE_BF16 ? 2 : 4; }
+
+// Bytes of partial sums the projection of n machines needs (largest group of a pass).
+size_t partial_bytes(const core_ctx *ctx, int32_t n, int64_t d, int dtype) {
+    size_t need = 0;
+    for (int32_t i0 = 0; i0 < n; i0 += kMaxGroup) {
+        const int32_t ng = n - i0 < kMaxGroup ? n - i0 : kMaxGroup;
+        const ProjectPlan plan = make_project_plan(ng, ctx->m, d, dtype, ctx->sm_count);
+        const size_t b = (size_t)plan.grid_x * ng * ctx->m * sizeof(float);
+        if (b > need) need = b;
+    }
+    return round_up(need, 256);
+}
+
+// Projects rows [0, n) of a matrix whose coordinate 0 is global block q_base; the partial
+// sums go through `partial`; P (n*m) receives (or accumulates) the result.
+int project_into(core_ctx *ctx, const void *G, int dtype, int32_t n, int64_t ldg, int64_t d, uint64_t q_base,
+                 float *partial, float *P, bool accumulate, cudaStream_t stream) {
+    for (int32_t i0 = 0; i0 < n; i0 += kMaxGroup) {
+        const int32_t ng = n - i0 < kMaxGroup ? n - i0 : kMaxGroup;
+        const ProjectPlan plan = make_project_plan(ng, ctx->m, d, dtype, ctx->sm_count);
+        const char *rows = static_cast<const char *>(G) + (size_t)i0 * (size_t)ldg * elem_size(dtype);
+        CORE_CUDA(ctx, launch_project(plan, ctx->keys, ctx->t, rows, dtype, ng, ldg, d, ctx->m, q_base, partial,
+                                      stream));
+        CORE_CUDA(ctx, launch_finish_project(partial, plan.grid_x, ng, ctx->m, P + (size_t)i0 * ctx->m, accumulate,
+                                             stream));
+    }
+    return CORE_OK;
+}
+
+int check_ctx(const core_ctx *ctx) {
+    if (!ctx) return CORE_EINVAL;
+    if (!on_device(ctx->device)) return CORE_EINVAL;
+    return CORE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int core_init(core_ctx **out, uint64_t seed, int64_t d, int32_t m) {
+    if (!out) return CORE_EINVAL;
+    *out = nullptr;
+    if (d < 1 || m < 1) return CORE_EINVAL;
+    core_ctx *ctx = new (std::nothrow) core_ctx();
+    if (!ctx) return CORE_ENOMEM;
+    ctx->seed = seed;
+    ctx->d = d;
+    ctx->m = m;
+    ctx->t = 0;
+    ctx->stream = nullptr;
+    ctx->keys = expand_keys(seed);
+    ctx->ws = nullptr;
+    ctx->ws_bytes = 0;
+    ctx->pbar = nullptr;
+    ctx->last_cuda = 0;
+    ctx->host_ready = false;
+    ctx->slab = nullptr;
+    ctx->slab_bytes = 0;
+    cudaError_t e = cudaGetDevice(&ctx->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->pbar), (size_t)m * sizeof(float));
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        const int rc = e == cudaErrorMemoryAllocation ? CORE_ENOMEM : CORE_ECUDA;
+        delete ctx;
+        return rc;
+    }
+    *out = ctx;
+    return CORE_OK;
+}
+
+int core_destroy(core_ctx *ctx) {
+    if (!ctx) return CORE_EINVAL;
+    int rc = CORE_OK;
+    if (ctx->ws && cudaFree(ctx->ws) != cudaSuccess) rc = CORE_ECUDA;
+    if (ctx->pbar && cudaFree(ctx->pbar) != cudaSuccess) rc = CORE_ECUDA;
+    if (ctx->slab && cudaFree(ctx->slab) != cudaSuccess) rc = CORE_ECUDA;
+    if (ctx->host_ready) {
+        cudaStreamDestroy(ctx->copy_stream);
+        cudaStreamDestroy(ctx->work_stream);
+        for (int s = 0; s < 2; ++s) {
+            cudaEventDestroy(ctx->in_ready[s]);
+            cudaEventDestroy(ctx->in_free[s]);
+            cudaEventDestroy(ctx->out_ready[s]);
+            cudaEventDestroy(ctx->out_free[s]);
+        }
+    }
+    delete ctx;
+    return rc;
+}
+
+int core_set_stream(core_ctx *ctx, void *cuda_stream) {
+    if (!ctx) return CORE_EINVAL;
+    ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    return CORE_OK;
+}
+
+int core_set_round(core_ctx *ctx, uint32_t t) {
+    if (!ctx) return CORE_EINVAL;
+    ctx->t = t;
+    return CORE_OK;
+}
+
+uint32_t core_get_round(const core_ctx *ctx) { return ctx ? ctx->t : 0u; }
+
+size_t core_workspace_bytes(const core_ctx *ctx) {
+    return ctx ? ctx->ws_bytes + ctx->slab_bytes + (size_t)ctx->m * sizeof(float) : 0;
+}
+
+const char *core_strerror(int code) {
+    switch (code) {
+        case CORE_OK: return "ok";
+        case CORE_EINVAL: return "invalid argument";
+        case CORE_ENOMEM: return "out of device memory";
+        case CORE_ECUDA: return "CUDA runtime error";
+        default: return "unknown error";
+    }
+}
+
+int core_last_cuda_error(const core_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }
+
+int core_project(core_ctx *ctx, const void *G_dev, int dtype, int32_t n, int64_t ldg, float *P_dev) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!G_dev || !P_dev || n < 1 || ldg < ctx->d || !valid_dtype(dtype)) return CORE_EINVAL;
+    if (int rc = ensure_workspace(ctx, partial_bytes(ctx, n, ctx->d, dtype))) return rc;
+    return project_into(ctx, G_dev, dtype, n, ldg, ctx->d, 0, static_cast<float *>(ctx->ws), P_dev, false,
+                        ctx->stream);
+}
+
+int core_aggregate(core_ctx *ctx, const float *P_dev, int32_t n, float *pbar_dev) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!P_dev || !pbar_dev || n < 1) return CORE_EINVAL;
+    CORE_CUDA(ctx, launch_aggregate(P_dev, n, ctx->m, pbar_dev, ctx->stream));
+    return CORE_OK;
+}
+
+int core_reconstruct(core_ctx *ctx, const float *pbar_dev, float *gtilde_dev) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!pbar_dev || !gtilde_dev) return CORE_EINVAL;
+    CORE_CUDA(ctx, launch_reconstruct(ctx->keys, ctx->t, pbar_dev, ctx->m, 0, ctx->d, gtilde_dev, ctx->sm_count,
+                                      ctx->stream));
+    return CORE_OK;
+}
+
+int core_round(core_ctx *ctx, const void *G_dev, int dtype, int32_t n, int64_t ldg, float *pbar_dev,
+               float *gtilde_dev) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!G_dev || !pbar_dev || !gtilde_dev || n < 1 || ldg < ctx->d || !valid_dtype(dtype)) return CORE_EINVAL;
+    const size_t pb = partial_bytes(ctx, n, ctx->d, dtype);
+    const size_t Pb = round_up((size_t)n * ctx->m * sizeof(float), 256);
+    if (int rc = ensure_workspace(ctx, pb + Pb)) return rc;
+    float *partial = static_cast<float *>(ctx->ws);
+    float *P = reinterpret_cast<float *>(static_cast<char *>(ctx->ws) + pb);
+    if (int rc = project_into(ctx, G_dev, dtype, n, ldg, ctx->d, 0, partial, P, false, ctx->stream)) return rc;
+    CORE_CUDA(ctx, launch_aggregate(P, n, ctx->m, pbar_dev, ctx->stream));
+    CORE_CUDA(ctx, launch_reconstruct(ctx->keys, ctx->t, pbar_dev, ctx->m, 0, ctx->d, gtilde_dev, ctx->sm_count,
+                                      ctx->stream));
+    ctx->t += 1;
+    return CORE_OK;
+}
+
+int core_round_host(core_ctx *ctx, const void *G_host, int dtype, int32_t n, int64_t ldg, float *pbar_host,
+                    float *gtilde_host) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!G_host || !pbar_host || !gtilde_host || n < 1 || ldg < ctx->d || !valid_dtype(dtype)) return CORE_EINVAL;
+    if (!ctx->host_ready) {
+        CORE_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+        CORE_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->work_stream, cudaStreamNonBlocking));
+        for (int s = 0; s < 2; ++s) {
+            CORE_CUDA(ctx, cudaEventCreateWithFlags(&ctx->in_ready[s], cudaEventDisableTiming));
+            CORE_CUDA(ctx, cudaEventCreateWithFlags(&ctx->in_free[s], cudaEventDisableTiming));
+            CORE_CUDA(ctx, cudaEventCreateWithFlags(&ctx->out_ready[s], cudaEventDisableTiming));
+            CORE_CUDA(ctx, cudaEventCreateWithFlags(&ctx->out_free[s], cudaEventDisableTiming));
+        }
+        ctx->host_ready = true;
+    }
+    const size_t es = elem_size(dtype);
+    const int64_t d = ctx->d;
+    // slab: a multiple of 4096 coordinates, about 64 MiB of input per slab over all machines
+    int64_t slab = ((int64_t)64 << 20) / (int64_t)(es * (size_t)n);
+    slab = slab / 4096 * 4096;
+    if (slab < 4096) slab = 4096;
+    if (slab > (d + 4095) / 4096 * 4096) slab = (d + 4095) / 4096 * 4096;
+    const size_t in_bytes = round_up((size_t)n * (size_t)slab * es, 256);
+    const size_t out_bytes = round_up((size_t)slab * sizeof(float), 256);
+    const size_t need_slab = 2 * in_bytes + 2 * out_bytes;
+    if (need_slab > ctx->slab_bytes) {
+        if (ctx->slab) {
+            cudaFree(ctx->slab);
+            ctx->slab = nullptr;
+            ctx->slab_bytes = 0;
+        }
+        cudaError_t e = cudaMalloc(&ctx->slab, need_slab);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            ctx->last_cuda = (int)e;
+            return CORE_ENOMEM;
+        }
+        ctx->slab_bytes = need_slab;
+    }
+    const size_t pb = partial_bytes(ctx, n, slab, dtype);
+    const size_t Pb = round_up((size_t)n * ctx->m * sizeof(float), 256);
+    const size_t mb = round_up((size_t)ctx->m * sizeof(float), 256);
+    if (int rc = ensure_workspace(ctx, pb + Pb + mb)) return rc;
+    char *in_buf[2] = {static_cast<char *>(ctx->slab), static_cast<char *>(ctx->slab) + in_bytes};
+    float *out_buf[2] = {reinterpret_cast<float *>(static_cast<char *>(ctx->slab) + 2 * in_bytes),
+                         reinterpret_cast<float *>(static_cast<char *>(ctx->slab) + 2 * in_bytes + out_bytes)};
+    float *partial = static_cast<float *>(ctx->ws);
+    float *P = reinterpret_cast<float *>(static_cast<char *>(ctx->ws) + pb);
+    float *pbar = reinterpret_cast<float *>(static_cast<char *>(ctx->ws) + pb + Pb);
+
+    CORE_CUDA(ctx, cudaStreamSynchronize(ctx->stream));   // earlier work of the caller on this context
+
+    // projection: slab s is copied while slab s-1 is projected
+    const int64_t slabs = (d + slab - 1) / slab;
+    for (int64_t s = 0; s < slabs; ++s) {
+        const int b = (int)(s & 1);
+        const int64_t k0 = s * slab;
+        const int64_t len = d - k0 < slab ? d - k0 : slab;
+        if (s >= 2) CORE_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->in_free[b], 0));
+        for (int32_t i = 0; i < n; ++i)   // one copy per row: row strides may exceed the 2-D copy pitch limit
+            CORE_CUDA(ctx, cudaMemcpyAsync(in_buf[b] + (size_t)i * (size_t)slab * es,
+                                           static_cast<const char *>(G_host) + ((size_t)i * (size_t)ldg + (size_t)k0) * es,
+                                           (size_t)len * es, cudaMemcpyHostToDevice, ctx->copy_stream));
+        CORE_CUDA(ctx, cudaEventRecord(ctx->in_ready[b], ctx->copy_stream));
+        CORE_CUDA(ctx, cudaStreamWaitEvent(ctx->work_stream, ctx->in_ready[b], 0));
+        if (int rc = project_into(ctx, in_buf[b], dtype, n, slab, len, (uint64_t)k0 >> 2, partial, P, s > 0,
+                                  ctx->work_stream))
+            return rc;
+        CORE_CUDA(ctx, cudaEventRecord(ctx->in_free[b], ctx->work_stream));
+    }
+    CORE_CUDA(ctx, launch_aggregate(P, n, ctx->m, pbar, ctx->work_stream));
+    CORE_CUDA(ctx, cudaMemcpyAsync(pbar_host, pbar, (size_t)ctx->m * sizeof(float), cudaMemcpyDeviceToHost,
+                                   ctx->work_stream));
+    // reconstruction: slab s is copied back while slab s+1 is generated
+    for (int64_t s = 0; s < slabs; ++s) {
+        const int b = (int)(s & 1);
+        const int64_t k0 = s * slab;
+        const int64_t len = d - k0 < slab ? d - k0 : slab;
+        if (s >= 2) CORE_CUDA(ctx, cudaStreamWaitEvent(ctx->work_stream, ctx->out_free[b], 0));
+        CORE_CUDA(ctx, launch_reconstruct(ctx->keys, ctx->t, pbar, ctx->m, k0, k0 + len, out_buf[b], ctx->sm_count,
+                                          ctx->work_stream));
+        CORE_CUDA(ctx, cudaEventRecord(ctx->out_ready[b], ctx->work_stream));
+        CORE_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->out_ready[b], 0));
+        CORE_CUDA(ctx, cudaMemcpyAsync(gtilde_host + k0, out_buf[b], (size_t)len * sizeof(float),
+                                       cudaMemcpyDeviceToHost, ctx->copy_stream));
+        CORE_CUDA(ctx, cudaEventRecord(ctx->out_free[b], ctx->copy_stream));
+    }
+    CORE_CUDA(ctx, cudaStreamSynchronize(ctx->work_stream));
+    CORE_CUDA(ctx, cudaStreamSynchronize(ctx->copy_stream));
+    ctx->t += 1;
+    return CORE_OK;
+}
+
+/* ---- least squares ---------------------------------------------------------- */
+
+int core_ls_create(core_ls **out, const float *A_dev, const float *b_dev, int32_t n, int32_t rows, int64_t d) {
+    if (!out) return CORE_EINVAL;
+    *out = nullptr;
+    if (!A_dev || !b_dev || n < 1 || rows < 1 || d < 1) return CORE_EINVAL;
+    core_ls *ls = new (std::nothrow) core_ls();
+    if (!ls) return CORE_ENOMEM;
+    ls->A = A_dev;
+    ls->b = b_dev;
+    ls->n = n;
+    ls->rows = rows;
+    ls->d = d;
+    int sm = 0;
+    cudaError_t e = cudaGetDevice(&ls->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, ls->device);
+    if (e != cudaSuccess) {
+        delete ls;
+        return CORE_ECUDA;
+    }
+    ls->plan = make_ls_plan(n, rows, d, sm);
+    const size_t res_b = round_up((size_t)n * rows * sizeof(float), 256);
+    const size_t part_b = round_up((size_t)n * ls->plan.splits * (size_t)d * sizeof(float), 256);
+    const size_t G_b = round_up((size_t)n * (size_t)d * sizeof(float), 256);
+    const size_t gt_b = round_up((size_t)d * sizeof(float), 256);
+    char *base = nullptr;
+    e = cudaMalloc(reinterpret_cast<void **>(&base), res_b + part_b + G_b + gt_b);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        delete ls;
+        return CORE_ENOMEM;
+    }
+    ls->res = reinterpret_cast<float *>(base);
+    ls->part = reinterpret_cast<float *>(base + res_b);
+    ls->G = reinterpret_cast<float *>(base + res_b + part_b);
+    ls->gt = reinterpret_cast<float *>(base + res_b + part_b + G_b);
+    *out = ls;
+    return CORE_OK;
+}
+
+int core_ls_destroy(core_ls *ls) {
+    if (!ls) return CORE_EINVAL;
+    const int rc = cudaFree(ls->res) == cudaSuccess ? CORE_OK : CORE_ECUDA;   // res is the base of the block
+    delete ls;
+    return rc;
+}
+
+static int ls_gradients_into(core_ctx *ctx, core_ls *ls, const float *x_dev, float *G) {
+    CORE_CUDA(ctx, launch_ls_residual(ls->A, ls->b, x_dev, ls->n, ls->rows, ls->d, ls->res, ctx->stream));
+    CORE_CUDA(ctx, launch_ls_at_r(ls->plan, ls->A, ls->res, ls->n, ls->rows, ls->d, ls->part, ctx->stream));
+    CORE_CUDA(ctx, launch_ls_reduce(ls->plan, ls->part, ls->n, ls->rows, ls->d, G, ctx->stream));
+    return CORE_OK;
+}
+
+int core_ls_gradients(core_ctx *ctx, core_ls *ls, const float *x_dev, float *G_out_dev) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!ls || !x_dev || !G_out_dev || ls->d != ctx->d || ls->device != ctx->device) return CORE_EINVAL;
+    return ls_gradients_into(ctx, ls, x_dev, G_out_dev);
+}
+
+int core_gd_step(core_ctx *ctx, core_ls *ls, float h, float *x_dev) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!ls || !x_dev || ls->d != ctx->d || ls->device != ctx->device) return CORE_EINVAL;
+    if (int rc = ls_gradients_into(ctx, ls, x_dev, ls->G)) return rc;
+    if (int rc = core_round(ctx, ls->G, CORE_F32, ls->n, ls->d, ctx->pbar, ls->gt)) return rc;
+    CORE_CUDA(ctx, launch_axpy(x_dev, ls->gt, h, ls->d, ctx->stream));
+    return CORE_OK;
+}
+
+int core_ls_loss(core_ctx *ctx, core_ls *ls, const float *x_dev, double *loss_dev) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!ls || !x_dev || !loss_dev || ls->d != ctx->d || ls->device != ctx->device) return CORE_EINVAL;
+    CORE_CUDA(ctx, launch_ls_residual(ls->A, ls->b, x_dev, ls->n, ls->rows, ls->d, ls->res, ctx->stream));
+    CORE_CUDA(ctx, launch_ls_loss(ls->res, ls->n, ls->rows, loss_dev, ctx->stream));
+    return CORE_OK;
+}
+
+/* ---- generator windows -------------------------------------------------------- */
+
+int core_debug_philox(core_ctx *ctx, uint32_t j, uint64_t q0, int64_t nq, uint32_t *words_dev) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!words_dev || nq < 0 || (reinterpret_cast<uintptr_t>(words_dev) % 16) != 0) return CORE_EINVAL;
+    CORE_CUDA(ctx, launch_debug_philox(ctx->keys, ctx->t, j, q0, nq, words_dev, ctx->stream));
+    return CORE_OK;
+}
+
+int core_debug_gaussians(core_ctx *ctx, uint32_t j, uint64_t q0, int64_t nq, float *z_dev) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!z_dev || nq < 0 || (reinterpret_cast<uintptr_t>(z_dev) % 16) != 0) return CORE_EINVAL;
+    CORE_CUDA(ctx, launch_debug_gaussians(ctx->keys, ctx->t, j, q0, nq, z_dev, ctx->stream));
+    return CORE_OK;
+}
+
+int core_debug_box_muller(core_ctx *ctx, const uint32_t *words_dev, int64_t nb, float *z_dev) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!words_dev || !z_dev || nb < 0 || (reinterpret_cast<uintptr_t>(words_dev) % 16) != 0 ||
+        (reinterpret_cast<uintptr_t>(z_dev) % 16) != 0)
+        return CORE_EINVAL;
+    CORE_CUDA(ctx, launch_debug_box_muller(words_dev, nb, z_dev, ctx->stream));
+    return CORE_OK;
+}
+
+int core_debug_project_plan(int32_t n, int32_t m, int64_t d, int dtype, int32_t sm_count, int64_t out[10]) {
+    if (!out || n < 1 || m < 1 || d < 1 || sm_count < 1 || !valid_dtype(dtype)) return CORE_EINVAL;
+    const ProjectPlan p = make_project_plan(n < kMaxGroup ? n : kMaxGroup, m, d, dtype, sm_count);
+    const int64_t v[10] = {p.nb, p.jt, p.uq, p.tile_q, p.tj, p.tq, p.grid_x, p.grid_y, p.tiles, (int64_t)p.smem};
+    for (int i = 0; i < 10; ++i) out[i] = v[i];
+    return CORE_OK;
+}
+
+}  // extern "C"

@@ -55,18 +55,21 @@ cudaError_t launch_debug_gaussians(const RoundKeys &keys, uint32_t t, uint32_t j
                                    float *z, cudaStream_t stream);
 cudaError_t launch_debug_box_muller(const uint32_t *words, int64_t nb, float *z, cudaStream_t stream);
 
-// Least squares: each machine's rows are split over ctas_per_machine CTAs; every CTA
-// leaves a partial gradient and a partial sum of squared residuals.
+// Least squares.  Pass 1: res[i*rows + r] = A_i[r] . x - b_i[r].  Pass 2: the rows of a
+// machine are cut into `splits` ranges; part[(i*splits + s)*d + k] = sum over the rows of
+// range s of A_i[r][k] * res_i[r].  Reduce: G[i*d + k] = (1/rows) sum_s part[i][s][k].
 struct LsPlan {
-    int ctas_per_machine;
-    int rows_per_cta;
+    int splits;
+    int rows_per_split;
 };
 LsPlan make_ls_plan(int32_t n, int32_t rows, int64_t d, int sm_count);
-cudaError_t launch_ls_partial(const LsPlan &plan, const float *A, const float *b, const float *x, int32_t n,
-                              int32_t rows, int64_t d, float *part, double *res2, cudaStream_t stream);
+cudaError_t launch_ls_residual(const float *A, const float *b, const float *x, int32_t n, int32_t rows,
+                               int64_t d, float *res, cudaStream_t stream);
+cudaError_t launch_ls_at_r(const LsPlan &plan, const float *A, const float *res, int32_t n, int32_t rows,
+                           int64_t d, float *part, cudaStream_t stream);
 cudaError_t launch_ls_reduce(const LsPlan &plan, const float *part, int32_t n, int32_t rows, int64_t d,
                              float *G, cudaStream_t stream);
-cudaError_t launch_ls_loss(const LsPlan &plan, const double *res2, int32_t n, int32_t rows, double *loss,
-                           cudaStream_t stream);
+// loss[0] = (1/n) sum_i 1/(2 rows) sum_r res_i[r]^2, summed in double in a fixed order
+cudaError_t launch_ls_loss(const float *res, int32_t n, int32_t rows, double *loss, cudaStream_t stream);
 
 }  // namespace core
