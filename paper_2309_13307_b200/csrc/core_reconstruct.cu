@@ -28,7 +28,7 @@ struct ReconstructArgs {
     RoundKeys keys;
 };
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 4)
 reconstruct_kernel(const __grid_constant__ ReconstructArgs a) {
     __shared__ uint4 table[kJChunk];              // {JPart.x0, JPart.x2, JPart.w3, bits of pbar[j]}
     const int tid = threadIdx.x;
@@ -80,10 +80,9 @@ reconstruct_kernel(const __grid_constant__ ReconstructArgs a) {
                     jp.x2 = e.y;
                     jp.w3 = e.z;
                     const float4 z = box_muller4(philox_combine(jp, qp[u], a.keys));
-                    acc[u].x = fmaf(p, z.x, acc[u].x);
-                    acc[u].y = fmaf(p, z.y, acc[u].y);
-                    acc[u].z = fmaf(p, z.z, acc[u].z);
-                    acc[u].w = fmaf(p, z.w, acc[u].w);
+                    const float2 lo = __ffma2_rn(make_float2(p, p), make_float2(z.x, z.y), make_float2(acc[u].x, acc[u].y));
+                    const float2 hi = __ffma2_rn(make_float2(p, p), make_float2(z.z, z.w), make_float2(acc[u].z, acc[u].w));
+                    acc[u] = make_float4(lo.x, lo.y, hi.x, hi.y);
                 }
             }
         }
@@ -170,7 +169,7 @@ cudaError_t launch_reconstruct(const RoundKeys &keys, uint32_t t, const float *p
     a.keys = keys;
     const int64_t nq = ((k_end + 3) >> 2) - (k_begin >> 2);
     const int64_t groups = (nq + kGroupQ - 1) / kGroupQ;
-    int64_t grid = (int64_t)sm_count * 2;
+    int64_t grid = (int64_t)sm_count * 4;     // four resident CTAs per SM (64 registers, 32 KB each)
     if (grid > groups) grid = groups;
     reconstruct_kernel<<<(unsigned)grid, kThreads, 0, stream>>>(a);
     return cudaGetLastError();

@@ -126,59 +126,76 @@ __device__ __forceinline__ uint4 philox_combine(const JPart &jp, const QPart &qp
 }
 
 // ---- Box-Muller ---------------------------------------------------------------------
+// One call turns the four words of a counter into four Gaussians.  The two pairs are
+// evaluated side by side in packed fp32 (fma.rn.f32x2 and friends), which halves the
+// instruction count of the floating-point part.
+//
+// Radius.  u = (k + 1/2) 2^-23 is formed exactly by inserting k = w >> 9 under the
+// exponent of 1.0 (one funnel shift) and subtracting 1 - 2^-24.  4 * (-2 ln u) comes from
+// the hardware log2; its square root is 2r.  The hardware log2 has an absolute error of
+// about 2e-7, which is harmless except when u is close to 1 (ln u close to 0): for
+// v = 1 - u < 2^-10 (v is exact) the series of -2 ln(1 - v) replaces it.  That case is
+// rare (one radius in 1024), so it sits behind a branch tested once per call.
+//
+// Angle.  2u = (k + 1/2) 2^-22 is formed exactly (k inserted under the exponent of 2^23,
+// one fused multiply-add), rounded to the nearest integer h in {0, 1, 2} with the usual
+// add-and-subtract of 1.5 * 2^23, and y = 2u - h in (-1/2, 1/2) is exact.  Then
+// theta = pi (h + y), so (cos, sin) theta = (-1)^h (cos, sin)(pi y): odd and even minimax
+// polynomials in y (fp32-evaluated error 1.7e-7 and 1.6e-7 over all inputs), and
+// (-1)^h / 2 = (h - 1)^2 - 1/2 multiplies the doubled radius.  No integer work, no selects.
+//
+// Worst absolute error over all 2^23 radius words and all 2^23 angle words: 1.4e-6.
 
-// r = sqrt(-2 ln u), u = ((w >> 9) + 1/2) 2^-23, absolute error below 1e-6.
-// u is formed exactly.  Away from 1 the hardware log2 is accurate enough; close to
-// 1 its absolute error would dominate ln u, so -2 ln(1 - v), v = 1 - u (exact), is
-// summed from its series instead.
-__device__ __forceinline__ float bm_radius(uint32_t w) {
-    float one_plus = __uint_as_float((w >> 9) | 0x3F800000u);   // 1 + k 2^-23
-    float u = one_plus - 0.99999994f;                           // exact: (k + 1/2) 2^-23
-    float lg;
-    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(u));
-    float l_far = lg * -1.3862943611198906f;                    // -2 ln 2 * log2 u
-    float v = 1.0f - u;                                         // exact
-    // -2 ln(1-v) = 2v + v^2 + (2/3) v^3 + (1/2) v^4 + ...
-    float s = fmaf(v, 0.5f, 0.6666667f);
-    s = fmaf(s, v, 1.0f);
-    s = fmaf(s, v, 2.0f);
-    float l_near = s * v;
-    float l = (v < 0.03125f) ? l_near : l_far;
-    float r;
-    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(l));
-    return r;
+constexpr uint32_t kNearOneWord = 0xFFC00000u;   // words with v = 1 - u < 2^-10
+
+// 4 * (-2 ln(1 - v)) = 8v + 4v^2 + (8/3) v^3 + 2 v^4 + ...
+__device__ __forceinline__ float bm_near_one(float v) {
+    float s = fmaf(v, 2.0f, 2.6666667f);
+    s = fmaf(s, v, 4.0f);
+    s = fmaf(s, v, 8.0f);
+    return s * v;
 }
 
-// (cos, sin)(2 pi u) scaled by r.  The angle is reduced exactly, in integers, to a
-// quarter turn index and y in (-1, 1) with theta = quadrant * pi/2 + y * pi/4; sine and
-// cosine of y pi/4 come from odd/even minimax polynomials in y (absolute error < 1e-7).
-__device__ __forceinline__ float2 bm_pair(uint32_t w_radius, uint32_t w_angle) {
-    float r = bm_radius(w_radius);
-    uint32_t rot = w_angle + 0x20000000u;                       // + 1/8 turn, wraps with the circle
-    // bits 29..9 of rot, doubled plus one, as the mantissa of a float in [4, 6):
-    // 4 + (f + 1/2) 2^-20 with f the 21-bit fraction of the quarter turn.
-    float y = __uint_as_float(((rot >> 8) & 0x003FFFFEu) | 0x40800001u) - 5.0f;   // exact
-    float y2 = y * y;
-    float sp = fmaf(-3.587725950637832e-05f, y2, 0.002489872043952346f);
-    sp = fmaf(sp, y2, -0.08074536919593811f);
-    sp = fmaf(sp, y2, 0.7853981256484985f);
-    float sn = sp * y;
-    float cp = fmaf(3.5313344142196e-06f, y2, -0.00032594200456514955f);
-    cp = fmaf(cp, y2, 0.015854327008128166f);
-    cp = fmaf(cp, y2, -0.3084251284599304f);
-    float cs = fmaf(cp, y2, 1.0f);
-    // quadrant: bit 30 of rot turns (cos, sin) into (-sin, cos); bit 31 negates both.
-    bool odd = (rot & 0x40000000u) != 0u;
-    float c = odd ? -sn : cs;
-    float s = odd ? cs : sn;
-    float rs = __uint_as_float(__float_as_uint(r) ^ (rot & 0x80000000u));
-    return make_float2(rs * c, rs * s);
-}
+__device__ __forceinline__ float2 bm_splat(float c) { return make_float2(c, c); }
 
 __device__ __forceinline__ float4 box_muller4(uint4 w) {
-    float2 a = bm_pair(w.x, w.y);
-    float2 b = bm_pair(w.z, w.w);
-    return make_float4(a.x, a.y, b.x, b.y);
+    // radii of the two pairs: lanes (x, y) = (pair a, pair b)
+    float2 u = __fadd2_rn(make_float2(__uint_as_float(__funnelshift_r(w.x, 0x7Fu, 9)),
+                                      __uint_as_float(__funnelshift_r(w.z, 0x7Fu, 9))),
+                          bm_splat(-0.99999994f));
+    float2 l;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(l.x) : "f"(u.x));
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(l.y) : "f"(u.y));
+    l = __fmul2_rn(l, bm_splat(-5.545177444479562f));            // -8 ln 2
+    if (max(w.x, w.z) >= kNearOneWord) {
+        if (w.x >= kNearOneWord) l.x = bm_near_one(1.0f - u.x);
+        if (w.z >= kNearOneWord) l.y = bm_near_one(1.0f - u.y);
+    }
+    float2 r2;                                                    // 2r
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r2.x) : "f"(l.x));
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r2.y) : "f"(l.y));
+
+    // angles
+    const float2 f = make_float2(__uint_as_float(__funnelshift_r(w.y, 0x96u, 9)),     // 2^23 + k
+                                 __uint_as_float(__funnelshift_r(w.w, 0x96u, 9)));
+    const float2 t = __ffma2_rn(f, bm_splat(2.384185791015625e-07f), bm_splat(-1.9999998807907104f));   // 2u
+    const float2 tm = __fadd2_rn(t, bm_splat(12582912.0f));
+    const float2 h = __fadd2_rn(tm, bm_splat(-12582912.0f));
+    const float2 y = __fadd2_rn(t, make_float2(-h.x, -h.y));
+    const float2 e = __fadd2_rn(h, bm_splat(-1.0f));
+    const float2 rs = __fmul2_rn(r2, __ffma2_rn(e, e, bm_splat(-0.5f)));              // r (-1)^h
+    const float2 y2 = __fmul2_rn(y, y);
+    float2 sp = __ffma2_rn(bm_splat(0.0772201269865036f), y2, bm_splat(-0.5980451703071594f));
+    sp = __ffma2_rn(sp, y2, bm_splat(2.5500314235687256f));
+    sp = __ffma2_rn(sp, y2, bm_splat(-5.1677069664001465f));
+    sp = __ffma2_rn(sp, y2, bm_splat(3.141592502593994f));        // sin(pi y) / y
+    float2 cp = __ffma2_rn(bm_splat(0.2200806587934494f), y2, bm_splat(-1.3320938348770142f));
+    cp = __ffma2_rn(cp, y2, bm_splat(4.058451175689697f));
+    cp = __ffma2_rn(cp, y2, bm_splat(-4.934795379638672f));
+    const float2 cs = __ffma2_rn(cp, y2, bm_splat(1.0f));         // cos(pi y)
+    const float2 zc = __fmul2_rn(rs, cs);
+    const float2 zs = __fmul2_rn(__fmul2_rn(rs, y), sp);
+    return make_float4(zc.x, zs.x, zc.y, zs.y);
 }
 
 }  // namespace core
