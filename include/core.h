@@ -48,7 +48,8 @@ enum {
     CORE_OK = 0,
     CORE_EINVAL = -1, /* null pointer, non-positive size, ld < d, unknown dtype */
     CORE_ENOMEM = -2, /* workspace allocation failed */
-    CORE_ECUDA = -3   /* CUDA runtime error; code via core_last_cuda_error */
+    CORE_ECUDA = -3,  /* CUDA runtime error; code via core_last_cuda_error */
+    CORE_ELIMIT = -4  /* size beyond the fixed capacity of an allocation-free entry point */
 };
 
 enum { CORE_F32 = 0, CORE_BF16 = 1 };
@@ -130,6 +131,40 @@ int core_round(core_ctx *ctx, const void *G_dev, int dtype, int32_t n, int64_t l
  */
 int core_round_host(core_ctx *ctx, const void *G_host, int dtype, int32_t n, int64_t ldg,
                     float *pbar_host, float *gtilde_host);
+
+/*
+ * Projection without any device allocation (the paper has no counterpart: this entry point
+ * exists for the library's users, not for the method).
+ *
+ * Who needs it: callers that cannot call cudaMalloc -- an application whose memory pool has
+ * claimed the whole device, or code on a path where the allocator's implicit device-wide
+ * synchronisation is not allowed.  core_init and core_project obtain a workspace with
+ * cudaMalloc; this call takes no context and obtains nothing.  The per-CTA partial sums of
+ * the projection go to a fixed array of CORE_STATIC_SCRATCH_FLOATS floats (4 MiB) that is
+ * part of the library image: every GPU that loads the library holds it until the process
+ * exits.
+ *
+ * Computes P[i*m + j] = <g_i, xi_j> exactly as core_project does for the generator keyed by
+ * (seed, round t); arguments as for core_project, plus d, m, seed and t passed directly.
+ * cuda_stream: the stream to enqueue on (NULL: default stream); returns without
+ * synchronising.  cuda_error_out (may be NULL) receives the CUDA error code when the return
+ * value is CORE_ECUDA.
+ *
+ * Limits: n <= 16 and n*m <= CORE_STATIC_SCRATCH_FLOATS, otherwise CORE_ELIMIT and nothing is
+ * launched.  When the usual number of CTA columns does not fit the array, fewer columns are
+ * used: slower, and the result may differ from core_project's in the last bits (same bound
+ * against the exact value).
+ *
+ * The first call on a device looks up the array's device address (no allocation, no
+ * synchronisation of the device); make that first call outside any stream capture.
+ * All calls share the one array, which keeps the previous call's contents: nothing in it
+ * needs to start at zero (every entry is written before it is read within a call), but two
+ * calls whose kernels overlap on the GPU -- different streams, no dependency between them --
+ * race on it.  Calls on one stream, or ordered by events, are safe.
+ */
+#define CORE_STATIC_SCRATCH_FLOATS ((size_t)1 << 20)
+int core_project_static(uint64_t seed, uint32_t t, int64_t d, int32_t m, const void *G_dev, int dtype,
+                        int32_t n, int64_t ldg, float *P_dev, void *cuda_stream, int *cuda_error_out);
 
 /* ---- least-squares CORE-GD driver (Algorithm 2) ----------------------------- */
 

@@ -13,7 +13,8 @@ import torch
 
 from . import build as _build
 
-CORE_OK, CORE_EINVAL, CORE_ENOMEM, CORE_ECUDA = 0, -1, -2, -3
+CORE_OK, CORE_EINVAL, CORE_ENOMEM, CORE_ECUDA, CORE_ELIMIT = 0, -1, -2, -3, -4
+CORE_STATIC_SCRATCH_FLOATS = 1 << 20
 CORE_F32, CORE_BF16 = 0, 1
 
 _lib = None
@@ -44,6 +45,8 @@ _SIGNATURES = {
     "core_debug_philox": ([_c.c_void_p, _c.c_uint32, _c.c_uint64, _c.c_int64, _c.c_void_p], _c.c_int),
     "core_debug_gaussians": ([_c.c_void_p, _c.c_uint32, _c.c_uint64, _c.c_int64, _c.c_void_p], _c.c_int),
     "core_debug_box_muller": ([_c.c_void_p, _c.c_void_p, _c.c_int64, _c.c_void_p], _c.c_int),
+    "core_project_static": ([_c.c_uint64, _c.c_uint32, _c.c_int64, _c.c_int32, _c.c_void_p, _c.c_int, _c.c_int32,
+                             _c.c_int64, _c.c_void_p, _c.c_void_p, _c.POINTER(_c.c_int)], _c.c_int),
     "core_debug_project_plan": ([_c.c_int32, _c.c_int32, _c.c_int64, _c.c_int, _c.c_int32,
                                  _c.POINTER(_c.c_int64)], _c.c_int),
 }
@@ -115,6 +118,24 @@ def core_debug_project_plan(n: int, m: int, d: int, dtype: int = CORE_F32, sm_co
         raise CoreError(rc, "core_debug_project_plan")
     keys = ("nb", "jt", "uq", "tile_q", "tj", "tq", "grid_x", "grid_y", "tiles", "smem")
     return dict(zip(keys, (int(v) for v in out)))
+
+
+def core_project_static(seed: int, t: int, m: int, G_dev: torch.Tensor, P_dev: torch.Tensor,
+                        stream: torch.cuda.Stream | None = None) -> torch.Tensor:
+    """Projection for callers that must not allocate device memory (no context, no workspace):
+    P_dev (caller-allocated, [n, m] float32) receives <g_i, xi_j>.  This wrapper allocates nothing
+    either.  Raises CoreError with code CORE_ELIMIT when n > 16 or n*m exceeds the fixed scratch."""
+    ptr, code, n, ld = _rows(G_dev)
+    if not G_dev.is_cuda:
+        raise ValueError("G must be a CUDA tensor")
+    stream = stream if stream is not None else torch.cuda.current_stream()
+    cuda_err = ctypes.c_int(0)
+    rc = lib().core_project_static(int(seed), int(t), int(G_dev.shape[1]), int(m), ptr, code, n, ld,
+                                   _dev(P_dev, torch.float32, n * m), ctypes.c_void_p(stream.cuda_stream),
+                                   ctypes.byref(cuda_err))
+    if rc != CORE_OK:
+        raise CoreError(rc, "core_project_static", cuda_err.value)
+    return P_dev
 
 
 class Core:

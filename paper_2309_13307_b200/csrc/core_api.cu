@@ -199,6 +199,7 @@ const char *core_strerror(int code) {
         case CORE_EINVAL: return "invalid argument";
         case CORE_ENOMEM: return "out of device memory";
         case CORE_ECUDA: return "CUDA runtime error";
+        case CORE_ELIMIT: return "size exceeds the fixed capacity of this entry point";
         default: return "unknown error";
     }
 }
