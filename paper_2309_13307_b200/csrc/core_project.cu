@@ -3,7 +3,7 @@
 //
 // The common vectors xi_j are generated in registers and never stored.  A CTA owns a
 // contiguous range of coordinate tiles and a range of vectors.  Thread (jl, ql) keeps JT
-// vectors j = jbase + jl + v*tj fixed and walks the coordinate blocks ql*UQ, ql*UQ + tq*UQ, ...
+// (4, or 2 with 16 machines) vectors j = jbase + jl + v*tj fixed and walks the coordinate blocks ql*UQ, ql*UQ + tq*UQ, ...
 // of every tile: one Philox counter gives the four Gaussians of (block, vector), which
 // meet the NB machine gradients of that block read (as broadcasts) from shared memory.
 // The gradient tile is staged once per CTA and tile, so G is read from HBM once per
@@ -168,13 +168,15 @@ project_kernel(const __grid_constant__ ProjectArgs a) {
             for (int v = 0; v < JT; ++v) acc[i][v] = 0.f;
 
         for (int qq = ql * UQ; qq < TILE_Q; qq += tq * UQ) {
-            float4 z[UQ][JT];
+            uint4 w[UQ * JT];
 #pragma unroll
             for (int u = 0; u < UQ; ++u) {
                 const QPart qp = philox_qpart(q0_lo + (uint32_t)(qq + u), a.t, a.keys);
 #pragma unroll
-                for (int v = 0; v < JT; ++v) z[u][v] = box_muller4(philox_combine(jp[v], qp, a.keys));
+                for (int v = 0; v < JT; ++v) w[u * JT + v] = philox_combine(jp[v], qp, a.keys);
             }
+            float4 z[UQ * JT];
+            box_muller4xN<UQ * JT>(w, z);
 #pragma unroll
             for (int i = 0; i < NB; ++i) {
 #pragma unroll
@@ -182,11 +184,12 @@ project_kernel(const __grid_constant__ ProjectArgs a) {
                     const float4 g = cur[i * TILE_Q + qq + u];
 #pragma unroll
                     for (int v = 0; v < JT; ++v) {
+                        const float4 zz = z[u * JT + v];
                         float s = acc[i][v];
-                        s = fmaf(g.x, z[u][v].x, s);
-                        s = fmaf(g.y, z[u][v].y, s);
-                        s = fmaf(g.z, z[u][v].z, s);
-                        s = fmaf(g.w, z[u][v].w, s);
+                        s = fmaf(g.x, zz.x, s);
+                        s = fmaf(g.y, zz.y, s);
+                        s = fmaf(g.z, zz.z, s);
+                        s = fmaf(g.w, zz.w, s);
                         acc[i][v] = s;
                     }
                 }
@@ -264,8 +267,9 @@ ProjectPlan make_project_plan(int32_t n_group, int32_t m, int64_t d, int dtype, 
     ProjectPlan p{};
     p.nb = 1;
     while (p.nb < n_group) p.nb *= 2;
-    p.jt = 2;
-    p.uq = (p.nb >= 16) ? 1 : 2;
+    // four generator calls per thread step: 4 vectors x 1 block (fewer machines) or 2 x 1
+    p.jt = (p.nb >= 8) ? 2 : 4;
+    p.uq = (p.nb == 8) ? 2 : 1;
     p.tile_q = tile_q_for(p.nb);
     int want = (m + p.jt - 1) / p.jt;                 // threads needed across vectors
     int tj = 1;
@@ -309,9 +313,9 @@ cudaError_t launch_project(const ProjectPlan &plan, const RoundKeys &keys, uint3
     a.t = t;
     a.keys = keys;
     switch (plan.nb) {
-        case 1: return launch_typed<1, 2, 2>(plan, a, dtype, stream);
-        case 2: return launch_typed<2, 2, 2>(plan, a, dtype, stream);
-        case 4: return launch_typed<4, 2, 2>(plan, a, dtype, stream);
+        case 1: return launch_typed<1, 4, 1>(plan, a, dtype, stream);
+        case 2: return launch_typed<2, 4, 1>(plan, a, dtype, stream);
+        case 4: return launch_typed<4, 4, 1>(plan, a, dtype, stream);
         case 8: return launch_typed<8, 2, 2>(plan, a, dtype, stream);
         default: return launch_typed<16, 2, 1>(plan, a, dtype, stream);
     }

@@ -28,6 +28,39 @@ struct ReconstructArgs {
     RoundKeys keys;
 };
 
+constexpr int kRecJStep = 2;                      // vectors generated together per loop step
+
+// acc[u] += sum over JS consecutive table entries of pbar[j] * xi_j[block u], j ascending.
+template <int JS>
+__device__ __forceinline__ void rec_step(const uint4 *entries, const QPart (&qp)[kRecUQ], const RoundKeys &keys,
+                                         float4 (&acc)[kRecUQ]) {
+    uint4 w[JS * kRecUQ];
+    float p[JS];
+#pragma unroll
+    for (int s = 0; s < JS; ++s) {
+        const uint4 e = entries[s];
+        p[s] = __uint_as_float(e.w);
+        JPart jp;
+        jp.x0 = e.x;
+        jp.x2 = e.y;
+        jp.w3 = e.z;
+#pragma unroll
+        for (int u = 0; u < kRecUQ; ++u) w[s * kRecUQ + u] = philox_combine(jp, qp[u], keys);
+    }
+    float4 z[JS * kRecUQ];
+    box_muller4xN<JS * kRecUQ>(w, z);
+#pragma unroll
+    for (int s = 0; s < JS; ++s) {
+#pragma unroll
+        for (int u = 0; u < kRecUQ; ++u) {
+            const float4 zz = z[s * kRecUQ + u];
+            const float2 lo = __ffma2_rn(make_float2(p[s], p[s]), make_float2(zz.x, zz.y), make_float2(acc[u].x, acc[u].y));
+            const float2 hi = __ffma2_rn(make_float2(p[s], p[s]), make_float2(zz.z, zz.w), make_float2(acc[u].z, acc[u].w));
+            acc[u] = make_float4(lo.x, lo.y, hi.x, hi.y);
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 4)
 reconstruct_kernel(const __grid_constant__ ReconstructArgs a) {
     __shared__ uint4 table[kJChunk];              // {JPart.x0, JPart.x2, JPart.w3, bits of pbar[j]}
@@ -69,22 +102,10 @@ reconstruct_kernel(const __grid_constant__ ReconstructArgs a) {
                 have_table = true;
                 table_qhi = grp_qhi;
             }
-#pragma unroll 2
-            for (int jj = 0; jj < jn; ++jj) {
-                const uint4 e = table[jj];
-                const float p = __uint_as_float(e.w);
-#pragma unroll
-                for (int u = 0; u < kRecUQ; ++u) {
-                    JPart jp;
-                    jp.x0 = e.x;
-                    jp.x2 = e.y;
-                    jp.w3 = e.z;
-                    const float4 z = box_muller4(philox_combine(jp, qp[u], a.keys));
-                    const float2 lo = __ffma2_rn(make_float2(p, p), make_float2(z.x, z.y), make_float2(acc[u].x, acc[u].y));
-                    const float2 hi = __ffma2_rn(make_float2(p, p), make_float2(z.z, z.w), make_float2(acc[u].z, acc[u].w));
-                    acc[u] = make_float4(lo.x, lo.y, hi.x, hi.y);
-                }
-            }
+            // kRecJStep vectors x kRecUQ blocks are generated together (one near-one test for all)
+            int jj = 0;
+            for (; jj + kRecJStep <= jn; jj += kRecJStep) rec_step<kRecJStep>(table + jj, qp, a.keys, acc);
+            for (; jj < jn; ++jj) rec_step<1>(table + jj, qp, a.keys, acc);
         }
 
 #pragma unroll

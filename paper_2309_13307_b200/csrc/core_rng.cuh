@@ -80,7 +80,8 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t q_lo, uint32_t q_hi, uin
 // words 0,1 depend only on (j, q_hi), words 2,3 only on (q_lo, t).  Round 1 then
 // needs MulA * word0 (a function of j, q_hi) and MulB * word2 (a function of q_lo, t).
 // A kernel that keeps j fixed while q varies, or q fixed while j varies, evaluates
-// the invariant half once.
+// the invariant half once.  The 32x32->64 multiply is the scarcest resource of the
+// generator on this GPU (a quarter of the fp32 rate), so this saves real time.
 
 struct JPart {       // depends on (j, q_hi)
     uint32_t x0;     // loB(j) ^ a1: xored with hiB(word 2) gives word 0 after round 1
@@ -128,74 +129,109 @@ __device__ __forceinline__ uint4 philox_combine(const JPart &jp, const QPart &qp
 // ---- Box-Muller ---------------------------------------------------------------------
 // One call turns the four words of a counter into four Gaussians.  The two pairs are
 // evaluated side by side in packed fp32 (fma.rn.f32x2 and friends), which halves the
-// instruction count of the floating-point part.
+// instruction count of the floating-point part.  On this GPU the fp32 pipe also executes
+// the wide multiplies of Philox, so the split of the work between pipes matters: bit
+// manipulation (integer pipe) is preferred over floating-point arithmetic where both can
+// do the job.
 //
 // Radius.  u = (k + 1/2) 2^-23 is formed exactly by inserting k = w >> 9 under the
-// exponent of 1.0 (one funnel shift) and subtracting 1 - 2^-24.  4 * (-2 ln u) comes from
-// the hardware log2; its square root is 2r.  The hardware log2 has an absolute error of
-// about 2e-7, which is harmless except when u is close to 1 (ln u close to 0): for
-// v = 1 - u < 2^-10 (v is exact) the series of -2 ln(1 - v) replaces it.  That case is
-// rare (one radius in 1024), so it sits behind a branch tested once per call.
+// exponent of 1.0 (one funnel shift) and subtracting 1 - 2^-24.  S = sqrt(-log2 u) comes
+// from the hardware log2 and square root; r = sqrt(2 ln 2) S, and that constant is folded
+// into the sine/cosine polynomials.  The hardware log2 has an absolute error of about
+// 2e-7, harmless except when u is close to 1 (log u close to 0): for v = 1 - u < 2^-10
+// (v is exact) the series of -log2(1 - v) replaces it.  That case is rare (one radius in
+// 1024), so it sits behind a branch tested once per call.
 //
-// Angle.  2u = (k + 1/2) 2^-22 is formed exactly (k inserted under the exponent of 2^23,
-// one fused multiply-add), rounded to the nearest integer h in {0, 1, 2} with the usual
-// add-and-subtract of 1.5 * 2^23, and y = 2u - h in (-1/2, 1/2) is exact.  Then
-// theta = pi (h + y), so (cos, sin) theta = (-1)^h (cos, sin)(pi y): odd and even minimax
-// polynomials in y (fp32-evaluated error 1.7e-7 and 1.6e-7 over all inputs), and
-// (-1)^h / 2 = (h - 1)^2 - 1/2 multiplies the doubled radius.  No integer work, no selects.
+// Angle.  theta = 2 pi u = pi (h + y): adding a quarter turn to the word (an integer add
+// that wraps with the circle) puts the parity of h = round(2u) in bit 31 and the 22
+// fraction bits of y + 1/2 in bits 30..9.  Those bits, doubled plus one, inserted under
+// the exponent of 1.0, minus 1.5, are y in (-1/2, 1/2) exactly.  Then
+// (cos, sin) theta = (-1)^h (cos, sin)(pi y): odd/even minimax polynomials in y, and bit 31
+// is xored into the sign of S.
 //
-// Worst absolute error over all 2^23 radius words and all 2^23 angle words: 1.4e-6.
+// Worst absolute error over all 2^23 radius words and all 2^23 angle words: 1.2e-6.
 
 constexpr uint32_t kNearOneWord = 0xFFC00000u;   // words with v = 1 - u < 2^-10
 
-// 4 * (-2 ln(1 - v)) = 8v + 4v^2 + (8/3) v^3 + 2 v^4 + ...
+// -log2(1 - v) = (v + v^2/2 + v^3/3 + v^4/4 + ...) / ln 2
 __device__ __forceinline__ float bm_near_one(float v) {
-    float s = fmaf(v, 2.0f, 2.6666667f);
-    s = fmaf(s, v, 4.0f);
-    s = fmaf(s, v, 8.0f);
+    float s = fmaf(v, 0.36067376f, 0.48089835f);
+    s = fmaf(s, v, 0.72134752f);
+    s = fmaf(s, v, 1.44269504f);
     return s * v;
 }
 
 __device__ __forceinline__ float2 bm_splat(float c) { return make_float2(c, c); }
 
-__device__ __forceinline__ float4 box_muller4(uint4 w) {
-    // radii of the two pairs: lanes (x, y) = (pair a, pair b)
-    float2 u = __fadd2_rn(make_float2(__uint_as_float(__funnelshift_r(w.x, 0x7Fu, 9)),
-                                      __uint_as_float(__funnelshift_r(w.z, 0x7Fu, 9))),
-                          bm_splat(-0.99999994f));
+// -log2 u of the two radius words of a call (lanes x, y = pair a, pair b) by the hardware
+// log2; u itself is returned for the rare correction.
+__device__ __forceinline__ float2 bm_neg_log2(uint4 w, float2 &u) {
+    u = __fadd2_rn(make_float2(__uint_as_float(__funnelshift_r(w.x, 0x7Fu, 9)),
+                               __uint_as_float(__funnelshift_r(w.z, 0x7Fu, 9))),
+                   bm_splat(-0.99999994f));
     float2 l;
     asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(l.x) : "f"(u.x));
     asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(l.y) : "f"(u.y));
-    l = __fmul2_rn(l, bm_splat(-5.545177444479562f));            // -8 ln 2
-    if (max(w.x, w.z) >= kNearOneWord) {
-        if (w.x >= kNearOneWord) l.x = bm_near_one(1.0f - u.x);
-        if (w.z >= kNearOneWord) l.y = bm_near_one(1.0f - u.y);
-    }
-    float2 r2;                                                    // 2r
-    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r2.x) : "f"(l.x));
-    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r2.y) : "f"(l.y));
+    return make_float2(-l.x, -l.y);
+}
+
+__device__ __forceinline__ void bm_fix_near_one(uint4 w, float2 u, float2 &l) {
+    if (w.x >= kNearOneWord) l.x = bm_near_one(1.0f - u.x);
+    if (w.z >= kNearOneWord) l.y = bm_near_one(1.0f - u.y);
+}
+
+// The rest of Box-Muller given l = -log2 u of the two pairs.
+__device__ __forceinline__ float4 bm_finish(uint4 w, float2 l) {
+    float2 s;
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(s.x) : "f"(l.x));
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(s.y) : "f"(l.y));
 
     // angles
-    const float2 f = make_float2(__uint_as_float(__funnelshift_r(w.y, 0x96u, 9)),     // 2^23 + k
-                                 __uint_as_float(__funnelshift_r(w.w, 0x96u, 9)));
-    const float2 t = __ffma2_rn(f, bm_splat(2.384185791015625e-07f), bm_splat(-1.9999998807907104f));   // 2u
-    const float2 tm = __fadd2_rn(t, bm_splat(12582912.0f));
-    const float2 h = __fadd2_rn(tm, bm_splat(-12582912.0f));
-    const float2 y = __fadd2_rn(t, make_float2(-h.x, -h.y));
-    const float2 e = __fadd2_rn(h, bm_splat(-1.0f));
-    const float2 rs = __fmul2_rn(r2, __ffma2_rn(e, e, bm_splat(-0.5f)));              // r (-1)^h
+    const uint32_t ra = w.y + 0x40000000u, rb = w.w + 0x40000000u;
+    const float2 y = __fadd2_rn(make_float2(__uint_as_float(((ra >> 8) & 0x007FFFFEu) | 0x3F800001u),
+                                            __uint_as_float(((rb >> 8) & 0x007FFFFEu) | 0x3F800001u)),
+                                bm_splat(-1.5f));
+    s.x = __uint_as_float(__float_as_uint(s.x) ^ (ra & 0x80000000u));
+    s.y = __uint_as_float(__float_as_uint(s.y) ^ (rb & 0x80000000u));
     const float2 y2 = __fmul2_rn(y, y);
-    float2 sp = __ffma2_rn(bm_splat(0.0772201269865036f), y2, bm_splat(-0.5980451703071594f));
-    sp = __ffma2_rn(sp, y2, bm_splat(2.5500314235687256f));
-    sp = __ffma2_rn(sp, y2, bm_splat(-5.1677069664001465f));
-    sp = __ffma2_rn(sp, y2, bm_splat(3.141592502593994f));        // sin(pi y) / y
-    float2 cp = __ffma2_rn(bm_splat(0.2200806587934494f), y2, bm_splat(-1.3320938348770142f));
-    cp = __ffma2_rn(cp, y2, bm_splat(4.058451175689697f));
-    cp = __ffma2_rn(cp, y2, bm_splat(-4.934795379638672f));
-    const float2 cs = __ffma2_rn(cp, y2, bm_splat(1.0f));         // cos(pi y)
-    const float2 zc = __fmul2_rn(rs, cs);
-    const float2 zs = __fmul2_rn(__fmul2_rn(rs, y), sp);
+    // sqrt(2 ln 2) sin(pi y) / y and sqrt(2 ln 2) cos(pi y)
+    float2 sp = __ffma2_rn(bm_splat(0.09091975539922714f), y2, bm_splat(-0.7041443586349487f));
+    sp = __ffma2_rn(sp, y2, bm_splat(3.0024325847625732f));
+    sp = __ffma2_rn(sp, y2, bm_splat(-6.08450984954834f));
+    sp = __ffma2_rn(sp, y2, bm_splat(3.6989426612854004f));
+    float2 cp = __ffma2_rn(bm_splat(0.2591251730918884f), y2, bm_splat(-1.568420648574829f));
+    cp = __ffma2_rn(cp, y2, bm_splat(4.778461456298828f));
+    cp = __ffma2_rn(cp, y2, bm_splat(-5.810277938842773f));
+    const float2 cs = __ffma2_rn(cp, y2, bm_splat(1.1774100065231323f));
+    const float2 zc = __fmul2_rn(s, cs);
+    const float2 zs = __fmul2_rn(__fmul2_rn(s, y), sp);
     return make_float4(zc.x, zs.x, zc.y, zs.y);
+}
+
+// N calls at once: the rare near-one correction of all 2N radii sits behind one test, which
+// leaves the N evaluations in one straight-line block for the instruction scheduler.
+template <int N>
+__device__ __forceinline__ void box_muller4xN(const uint4 (&w)[N], float4 (&z)[N]) {
+    float2 u[N], l[N];
+    uint32_t top = 0u;
+#pragma unroll
+    for (int c = 0; c < N; ++c) {
+        l[c] = bm_neg_log2(w[c], u[c]);
+        top = max(top, max(w[c].x, w[c].z));
+    }
+    if (top >= kNearOneWord) {
+#pragma unroll
+        for (int c = 0; c < N; ++c) bm_fix_near_one(w[c], u[c], l[c]);
+    }
+#pragma unroll
+    for (int c = 0; c < N; ++c) z[c] = bm_finish(w[c], l[c]);
+}
+
+__device__ __forceinline__ float4 box_muller4(uint4 w) {
+    const uint4 ws[1] = {w};
+    float4 zs[1];
+    box_muller4xN<1>(ws, zs);
+    return zs[0];
 }
 
 }  // namespace core
