@@ -29,12 +29,43 @@ if ROOT not in sys.path:
 METRIC = "CORE round throughput (coords x m projected+reconstructed/s)"
 UNIT = "coord*vector pairs/s"
 SEED_DATA, SEED_XI = 0, 1
-SM_COUNT, LANES_PER_SM = 148, 128
-# Algorithmic lane-operations per generated Gaussian: Philox4x32-10 = (20 wide multiplies +
-# 20 three-input xors) / 4 words = 10; Box-Muller per pair = 2 x (shift, or, add) to form the
-# uniforms' floats ... counted as 12 per pair = 6 per Gaussian.  Plus one FMA per machine
-# (project) or one FMA (reconstruct).
-OPS_PER_GAUSSIAN = 16
+SM_COUNT = 148
+# Philox4x32-10 multiplies two counter words by constants in each of ten rounds: 20 32x32->64-bit
+# multiplies per counter, and a counter yields four Gaussians.
+WIDE_MULS_PER_GAUSSIAN = 5
+# Measured on B200 with a dependent-chain microbenchmark: mul.wide.u32 retires 32 lanes per clock per SM
+# (one warp instruction per four clocks per scheduler), against 128 for fp32 FMA and 64 for logic ops.
+WIDE_MUL_LANES_PER_CLK_SM = 32
+
+
+def csrc_digest() -> str:
+    """sha256 over the CUDA sources: ties stored profiler counters to the code they were taken from."""
+    import glob
+    import hashlib
+    h = hashlib.sha256()
+    for path in sorted(glob.glob(os.path.join(ROOT, "paper_2309_13307_b200", "csrc", "*"))):
+        h.update(os.path.basename(path).encode())
+        h.update(open(path, "rb").read())
+    return h.hexdigest()
+
+
+def stored_traffic(kernel: str, d: int, m: int):
+    """DRAM bytes per launch from the committed ncu capture (profiles/round_kernels_dram.json), scaled by the
+    number of coordinates (traffic of both kernels is proportional to d); None if the kernels have changed
+    since the capture or no capture exists for this kernel."""
+    try:
+        rec = json.load(open(os.path.join(ROOT, "profiles", "round_kernels_dram.json")))
+    except (OSError, ValueError):
+        return None
+    if rec.get("csrc_sha256") != csrc_digest():
+        return None
+    best = None
+    for cap in rec.get("captures", []):
+        if cap["kernel"] == kernel and (best is None or abs(cap["m"] - m) < abs(best["m"] - m)):
+            best = cap
+    if best is None:
+        return None
+    return int(best["dram_bytes"] * (d / best["d"]))
 
 
 def parse_args():
@@ -297,24 +328,32 @@ def run_ours(args):
     except OSError:
         pass
     sm_max = (clocks or {}).get("sm_max_mhz") or peaks.get("sm_max_mhz") or 1965.0
-    alu_peak = SM_COUNT * LANES_PER_SM * sm_max * 1e6          # lane-operations per second
+    hbm_peak = peaks.get("hbm_gbs", 6650.0) * 1e9
+    hbm_src = "of measured" if "hbm_gbs" in peaks else "of fallback"
+    # The binding unit of both round kernels is the 32x32->64-bit integer multiplier: Philox4x32-10
+    # needs 20 wide multiplies per counter = 5 per Gaussian, and the multiplier retires
+    # WIDE_MUL_LANES_PER_CLK_SM of them per clock per SM (measured; a quarter of the fp32 rate).
+    wide_peak = SM_COUNT * WIDE_MUL_LANES_PER_CLK_SM * sm_max * 1e6        # wide multiplies per second
     kernels = []
     for m in ms:
         tp, ta, tr = per_m[m]
-        kernels.append(("project", m, tp, OPS_PER_GAUSSIAN + n, n * d * G.element_size()))
-        kernels.append(("reconstruct", m, tr, OPS_PER_GAUSSIAN + 1, 4 * d))
-    name, m_dom, t_dom, ops_per_unit, hbm_bytes = max(kernels, key=lambda k: k[2])
-    achieved = d * m_dom * ops_per_unit / (t_dom * 1e-3)
-    roofline = {"bound": "alu", "kernel": f"{name} m={m_dom}", "achieved": achieved / 1e12, "peak": alu_peak / 1e12,
-                "unit": "Tlane-op/s", "frac": achieved / alu_peak, "traffic": None,
-                "ops_per_unit": ops_per_unit, "ms_per_launch": t_dom,
-                "peak_source": f"148 SM x 128 fp32/int32 lanes x {sm_max:.0f} MHz (max SM clock)",
-                "hbm_frac_of_measured": (hbm_bytes / (t_dom * 1e-3)) / (peaks.get("hbm_gbs", 6650.0) * 1e9)}
+        kernels.append(("project", m, tp, n * d * G.element_size()))
+        kernels.append(("reconstruct", m, tr, 4 * d + 4 * m))
+    name, m_dom, t_dom, hbm_bytes = max(kernels, key=lambda k: k[2])
+    achieved = d * m_dom * WIDE_MULS_PER_GAUSSIAN / (t_dom * 1e-3)
+    roofline = {"bound": "alu", "kernel": f"{name} m={m_dom}", "achieved": achieved / 1e12, "peak": wide_peak / 1e12,
+                "unit": "T wide-multiply/s", "frac": achieved / wide_peak,
+                "traffic": stored_traffic(name, d, m_dom),
+                "algorithmic_bytes": hbm_bytes, "ms_per_launch": t_dom,
+                "peak_source": f"148 SM x {WIDE_MUL_LANES_PER_CLK_SM} wide multiplies/clk/SM (measured) x {sm_max:.0f} MHz "
+                               f"(max SM clock); {WIDE_MULS_PER_GAUSSIAN} wide multiplies per pair",
+                "pairs_per_s": d * m_dom / (t_dom * 1e-3), "peak_pairs_per_s": wide_peak / WIDE_MULS_PER_GAUSSIAN,
+                "hbm_frac": (hbm_bytes / (t_dom * 1e-3)) / hbm_peak, "hbm_peak": hbm_src}
     sweep = []
-    for kname, m, t_ms, ops, hb in kernels:
-        sweep.append({"kernel": kname, "m": m, "ms": round(t_ms, 4), "units_per_s": d * m / (t_ms * 1e-3),
-                      "alu_frac": d * m * ops / (t_ms * 1e-3) / alu_peak,
-                      "hbm_frac": hb / (t_ms * 1e-3) / (peaks.get("hbm_gbs", 6650.0) * 1e9)})
+    for kname, m, t_ms, hb in kernels:
+        sweep.append({"kernel": kname, "m": m, "ms": round(t_ms, 4), "pairs_per_s": d * m / (t_ms * 1e-3),
+                      "alu_frac": d * m * WIDE_MULS_PER_GAUSSIAN / (t_ms * 1e-3) / wide_peak,
+                      "hbm_frac": hb / (t_ms * 1e-3) / hbm_peak})
 
     cpu = None if args.no_cpu else cpu_baseline_sample()
     out = {

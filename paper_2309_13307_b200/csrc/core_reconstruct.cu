@@ -61,7 +61,7 @@ __device__ __forceinline__ void rec_step(const uint4 *entries, const QPart (&qp)
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 4)
+__global__ void __launch_bounds__(kThreads, 3)
 reconstruct_kernel(const __grid_constant__ ReconstructArgs a) {
     __shared__ uint4 table[kJChunk];              // {JPart.x0, JPart.x2, JPart.w3, bits of pbar[j]}
     const int tid = threadIdx.x;
@@ -190,7 +190,7 @@ cudaError_t launch_reconstruct(const RoundKeys &keys, uint32_t t, const float *p
     a.keys = keys;
     const int64_t nq = ((k_end + 3) >> 2) - (k_begin >> 2);
     const int64_t groups = (nq + kGroupQ - 1) / kGroupQ;
-    int64_t grid = (int64_t)sm_count * 4;     // four resident CTAs per SM (64 registers, 32 KB each)
+    int64_t grid = (int64_t)sm_count * 3;     // three resident CTAs per SM (register-limited)
     if (grid > groups) grid = groups;
     reconstruct_kernel<<<(unsigned)grid, kThreads, 0, stream>>>(a);
     return cudaGetLastError();
