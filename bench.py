@@ -206,6 +206,23 @@ def run_reference(args):
 
 # ---- GPU leg ---------------------------------------------------------------------------------
 
+def slowest_rank(seconds_or_ms: float, world: int, device) -> float:
+    """Maximum of a per-rank duration over all ranks (identity for one rank).  The replicas are
+    independent, so the job is as slow as its slowest rank."""
+    if world <= 1:
+        return seconds_or_ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([seconds_or_ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_throughput(units_per_step: int, steps: int, world: int, elapsed_ms: float) -> float:
+    """Pairs per second over all replicas: every rank processes units_per_step per step (weak scaling)."""
+    return world * units_per_step * steps / (elapsed_ms * 1e-3)
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -271,12 +288,8 @@ def run_ours(args):
     stop.record()
     barrier()
     clocks = sampler.stop() if rank == 0 else None
-    elapsed_ms = start.elapsed_time(stop)
-    if world > 1:
-        tmax = torch.tensor([elapsed_ms], device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tmax.item())
-    value = world * units_per_step * args.steps / (elapsed_ms * 1e-3)
+    elapsed_ms = slowest_rank(start.elapsed_time(stop), world, "cuda")
+    value = whole_job_throughput(units_per_step, args.steps, world, elapsed_ms)
 
     # per-kernel times (averages over the timed launches)
     per_m = {}
@@ -304,12 +317,8 @@ def run_ours(args):
             for m in ms:
                 ctxs[m].core_round_host(Gh, pbar_h[m], gt_h)
         torch.cuda.synchronize()
-        dt = time.perf_counter() - t0
-        if world > 1:
-            tt = torch.tensor([dt], device="cuda")
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            dt = float(tt.item())
-        e2e = {"value": world * units_per_step * e2e_steps / dt, "unit": UNIT,
+        dt = slowest_rank(time.perf_counter() - t0, world, "cuda")
+        e2e = {"value": whole_job_throughput(units_per_step, e2e_steps, world, dt * 1e3), "unit": UNIT,
                "h2d_bytes_per_step": len(ms) * n * d * G.element_size(),
                "d2h_bytes_per_step": len(ms) * (d * 4) + sum(ms) * 4,
                "steps": e2e_steps, "how": "core_round_host from pinned host buffers, host clock around the "
