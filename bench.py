@@ -76,6 +76,8 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--d", type=int, default=None, help="override the coordinate count (development)")
     ap.add_argument("--m", type=int, nargs="*", default=None, help="override the m sweep (development)")
+    ap.add_argument("--workload", default="sweep", choices=["sweep", "leastsq"],
+                    help="sweep: the headline CORE round; leastsq: the CORE-GD step (secondary line)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     return ap.parse_args()
@@ -380,10 +382,59 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_leastsq(args):
+    """Secondary line: the least-squares CORE-GD step (n=8 machines, A_i 2048 x 8192, m=64), which is bound by
+    the two streaming passes over A.  Not the headline metric; reported for the HBM roofline of that step."""
+    import torch
+
+    import core_inputs
+    import paper_2309_13307_b200 as core_mod
+
+    torch.cuda.set_device(0)
+    core_mod.lib()
+    ls_in = core_inputs.least_squares(n=8, rows=2048, d=8192, seed=SEED_DATA, device="cuda")
+    n, rows, d = ls_in.A.shape
+    m = 64
+    h = float(1.0 / core_inputs.lipschitz_constant(ls_in.A, iters=30))
+    ctx = core_mod.Core(SEED_XI, d, m)
+    ls = core_mod.LeastSquares(ls_in.A, ls_in.b)
+    x = torch.zeros(d, dtype=torch.float32, device="cuda")
+    steps = max(args.steps, 50)
+    for _ in range(max(args.warmup, 3)):
+        ctx.core_gd_step(ls, h, x)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        ctx.core_gd_step(ls, h, x)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except OSError:
+        pass
+    a_bytes = ls_in.A.numel() * 4
+    hbm_peak = peaks.get("hbm_gbs", 6650.0)
+    achieved = 2 * a_bytes / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": "least-squares CORE-GD step", "value": ms, "unit": "ms/step", "higher_is_better": False,
+        "n_gpus": 1, "steps": steps, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"leastsq: n={n}, A_i {rows}x{d} fp32 (|A| = {a_bytes} bytes, larger than L2), m={m}"},
+        "loss": float(ctx.core_ls_loss(ls, x).item()), "gpu_launches": 8 * steps,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
+                     "traffic": None, "algorithmic_bytes": 2 * a_bytes,
+                     "peak_source": "of measured" if "hbm_gbs" in peaks else "of fallback",
+                     "note": "whole step (two passes over A, the round at d=8192 and the update) against 2|A| bytes"}}))
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "leastsq":
+        run_leastsq(args)
     else:
         run_ours(args)
 

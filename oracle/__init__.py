@@ -80,6 +80,8 @@ def lib() -> ctypes.CDLL:
             L.oracle_ls_grad.restype = None
             L.oracle_gd_step.argtypes = [u64, u32, i32, vp, vp, i32, i32, i64, dbl, vp, vp, ci]
             L.oracle_gd_step.restype = None
+            L.oracle_agd_step.argtypes = [u64, u32, i32, vp, vp, i32, i32, i64, dbl, dbl, vp, vp, vp, ci]
+            L.oracle_agd_step.restype = None
             _lib = L
     return _lib
 
@@ -235,3 +237,15 @@ def gd_step(seed: int, t: int, m: int, A, b, h: float, x: np.ndarray, exact: boo
     lib().oracle_gd_step(seed, t, m, _ptr(A), _ptr(b), n, rows, d, float(h), _ptr(x), _ptr(work),
                          1 if exact else 0)
     return x
+
+
+def agd_step(seed: int, t: int, m: int, A, b, h: float, beta: float, x: np.ndarray, x_prev: np.ndarray,
+             exact: bool = False):
+    """One Algorithm-4 iteration with round index t; returns (x_new, x)."""
+    A, b, n, rows, d = _ls_arrays(A, b)
+    x = np.array(x, dtype=np.float64, copy=True)
+    x_prev = np.array(x_prev, dtype=np.float64, copy=True)
+    work = np.zeros(d + n * d + n * m + m + d, dtype=np.float64)
+    lib().oracle_agd_step(seed, t, m, _ptr(A), _ptr(b), n, rows, d, float(h), float(beta), _ptr(x), _ptr(x_prev),
+                          _ptr(work), 1 if exact else 0)
+    return x, x_prev

@@ -225,3 +225,20 @@ void oracle_gd_step(uint64_t seed, uint32_t t, int32_t m, const float *A, const 
     }
     for (int64_t k = 0; k < d; ++k) x[k] -= h * gt[k];
 }
+
+/* ---- Algorithm 4: CORE-AGD (heavy ball with the CORE gradient estimate) ------ */
+
+void oracle_agd_step(uint64_t seed, uint32_t t, int32_t m, const float *A, const float *b, int32_t n,
+                     int32_t rows, int64_t d, double h, double beta, double *x, double *x_prev,
+                     double *work, int exact) {
+    double *y = work; /* d doubles, then the gd-step work area */
+    double *rest = work + d;
+    /* look-ahead point y^k = x^k + (1 - beta)(x^k - x^{k-1}) */
+    for (int64_t k = 0; k < d; ++k) y[k] = x[k] + (1.0 - beta) * (x[k] - x_prev[k]);
+    /* x^{k+1} = y^k - h * gradient estimate at y^k: a CORE-GD step taken from y */
+    oracle_gd_step(seed, t, m, A, b, n, rows, d, h, y, rest, exact);
+    for (int64_t k = 0; k < d; ++k) {
+        x_prev[k] = x[k];
+        x[k] = y[k];
+    }
+}

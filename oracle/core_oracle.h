@@ -113,6 +113,16 @@ void oracle_ls_grad(const float *A, const float *b, int32_t n, int32_t rows, int
 void oracle_gd_step(uint64_t seed, uint32_t t, int32_t m, const float *A, const float *b, int32_t n,
                     int32_t rows, int64_t d, double h, double *x, double *work, int exact);
 
+/*
+ * One CORE-AGD iteration (Algorithm 4: heavy ball on top of the CORE estimate) with round
+ * index t: y = x + (1 - beta)(x - x_prev); x_new = y - h * gtilde(y); then x_prev <- x,
+ * x <- x_new.  The gradient is taken at y (the algorithm's title and update line say y; its
+ * displayed reconstruction formula prints x, a typo).  work: d doubles more than gd_step needs.
+ */
+void oracle_agd_step(uint64_t seed, uint32_t t, int32_t m, const float *A, const float *b, int32_t n,
+                     int32_t rows, int64_t d, double h, double beta, double *x, double *x_prev,
+                     double *work, int exact);
+
 #ifdef __cplusplus
 }
 #endif

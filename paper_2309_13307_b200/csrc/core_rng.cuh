@@ -163,16 +163,16 @@ __device__ __forceinline__ float bm_near_one(float v) {
 
 __device__ __forceinline__ float2 bm_splat(float c) { return make_float2(c, c); }
 
-// -log2 u of the two radius words of a call (lanes x, y = pair a, pair b) by the hardware
-// log2; u itself is returned for the rare correction.
-__device__ __forceinline__ float2 bm_neg_log2(uint4 w, float2 &u) {
+// log2 u (negative) of the two radius words of a call (lanes x, y = pair a, pair b) by the
+// hardware log2; u itself is returned for the rare correction.
+__device__ __forceinline__ float2 bm_log2(uint4 w, float2 &u) {
     u = __fadd2_rn(make_float2(__uint_as_float(__funnelshift_r(w.x, 0x7Fu, 9)),
                                __uint_as_float(__funnelshift_r(w.z, 0x7Fu, 9))),
                    bm_splat(-0.99999994f));
     float2 l;
     asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(l.x) : "f"(u.x));
     asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(l.y) : "f"(u.y));
-    return make_float2(-l.x, -l.y);
+    return l;
 }
 
 __device__ __forceinline__ void bm_fix_near_one(uint4 w, float2 u, float2 &l) {
@@ -180,11 +180,12 @@ __device__ __forceinline__ void bm_fix_near_one(uint4 w, float2 u, float2 &l) {
     if (w.z >= kNearOneWord) l.y = bm_near_one(1.0f - u.y);
 }
 
-// The rest of Box-Muller given l = -log2 u of the two pairs.
+// The rest of Box-Muller given l with |l| = -log2 u of the two pairs (the sign of l is ignored:
+// the hardware path delivers log2 u < 0, the correction delivers the positive series).
 __device__ __forceinline__ float4 bm_finish(uint4 w, float2 l) {
     float2 s;
-    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(s.x) : "f"(l.x));
-    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(s.y) : "f"(l.y));
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(s.x) : "f"(fabsf(l.x)));
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(s.y) : "f"(fabsf(l.y)));
 
     // angles
     const uint32_t ra = w.y + 0x40000000u, rb = w.w + 0x40000000u;
@@ -216,8 +217,8 @@ __device__ __forceinline__ void box_muller4xN(const uint4 (&w)[N], float4 (&z)[N
     uint32_t top = 0u;
 #pragma unroll
     for (int c = 0; c < N; ++c) {
-        l[c] = bm_neg_log2(w[c], u[c]);
-        top = max(top, max(w[c].x, w[c].z));
+        l[c] = bm_log2(w[c], u[c]);
+        top = __vimax3_u32(top, w[c].x, w[c].z);
     }
     if (top >= kNearOneWord) {
 #pragma unroll
