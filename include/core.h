@@ -182,9 +182,21 @@ int core_ls_destroy(core_ls *ls);
  * One iteration of Algorithm 2: g_i = A_i^T (A_i x - b_i) / rows for every
  * machine, one round with the context's current t (then t <- t + 1), and
  * x <- x - h * gtilde.  x_dev: d floats, updated in place.  ctx must have been
- * created with the same d.
+ * created with the same d.  The update is applied inside the reconstruction
+ * kernel; the estimate itself is not stored.
  */
 int core_gd_step(core_ctx *ctx, core_ls *ls, float h, float *x_dev);
+
+/*
+ * One iteration of CORE-AGD (the accelerated, heavy-ball variant in the paper's
+ * appendix "Acceleration of CORE-GD", Algorithm 4):
+ *   y = x + (1 - beta)(x - x_prev);  gtilde = one round on the machine gradients
+ *   at y (current t, then t <- t + 1);  x_prev <- x;  x <- y - h * gtilde.
+ * The gradient is taken at y, as the algorithm's update line states (its displayed
+ * reconstruction formula prints x).  x_dev, x_prev_dev: d floats each, distinct,
+ * both updated in place; for the first iteration pass x_prev = x.
+ */
+int core_agd_step(core_ctx *ctx, core_ls *ls, float h, float beta, float *x_dev, float *x_prev_dev);
 
 /* loss_dev[0] = f(x) as a double, computed on the device. */
 int core_ls_loss(core_ctx *ctx, core_ls *ls, const float *x_dev, double *loss_dev);

@@ -39,7 +39,7 @@ struct core_ls {
     float *res;          // n*rows
     float *part;         // n*splits*d
     float *G;            // n*d
-    float *gt;           // d
+    float *y;            // d: look-ahead point of the accelerated step
 };
 
 namespace {
@@ -229,10 +229,10 @@ int core_reconstruct(core_ctx *ctx, const float *pbar_dev, float *gtilde_dev) {
     return CORE_OK;
 }
 
-int core_round(core_ctx *ctx, const void *G_dev, int dtype, int32_t n, int64_t ldg, float *pbar_dev,
-               float *gtilde_dev) {
-    if (int rc = check_ctx(ctx)) return rc;
-    if (!G_dev || !pbar_dev || !gtilde_dev || n < 1 || ldg < ctx->d || !valid_dtype(dtype)) return CORE_EINVAL;
+// project -> aggregate -> reconstruct with the current t, then t <- t + 1.  With an epilogue the
+// reconstruction writes the optimiser update into `out` instead of the estimate.
+static int round_with_epilogue(core_ctx *ctx, const void *G_dev, int dtype, int32_t n, int64_t ldg, float *pbar_dev,
+                               float *out, const ReconstructEpilogue *epilogue) {
     const size_t pb = partial_bytes(ctx, n, ctx->d, dtype);
     const size_t Pb = round_up((size_t)n * ctx->m * sizeof(float), 256);
     if (int rc = ensure_workspace(ctx, pb + Pb)) return rc;
@@ -240,10 +240,17 @@ int core_round(core_ctx *ctx, const void *G_dev, int dtype, int32_t n, int64_t l
     float *P = reinterpret_cast<float *>(static_cast<char *>(ctx->ws) + pb);
     if (int rc = project_into(ctx, G_dev, dtype, n, ldg, ctx->d, 0, partial, P, false, ctx->stream)) return rc;
     CORE_CUDA(ctx, launch_aggregate(P, n, ctx->m, pbar_dev, ctx->stream));
-    CORE_CUDA(ctx, launch_reconstruct(ctx->keys, ctx->t, pbar_dev, ctx->m, 0, ctx->d, gtilde_dev, ctx->sm_count,
-                                      ctx->stream));
+    CORE_CUDA(ctx, launch_reconstruct(ctx->keys, ctx->t, pbar_dev, ctx->m, 0, ctx->d, out, ctx->sm_count, ctx->stream,
+                                      epilogue));
     ctx->t += 1;
     return CORE_OK;
+}
+
+int core_round(core_ctx *ctx, const void *G_dev, int dtype, int32_t n, int64_t ldg, float *pbar_dev,
+               float *gtilde_dev) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!G_dev || !pbar_dev || !gtilde_dev || n < 1 || ldg < ctx->d || !valid_dtype(dtype)) return CORE_EINVAL;
+    return round_with_epilogue(ctx, G_dev, dtype, n, ldg, pbar_dev, gtilde_dev, nullptr);
 }
 
 int core_round_host(core_ctx *ctx, const void *G_host, int dtype, int32_t n, int64_t ldg, float *pbar_host,
@@ -374,7 +381,7 @@ int core_ls_create(core_ls **out, const float *A_dev, const float *b_dev, int32_
     ls->res = reinterpret_cast<float *>(base);
     ls->part = reinterpret_cast<float *>(base + res_b);
     ls->G = reinterpret_cast<float *>(base + res_b + part_b);
-    ls->gt = reinterpret_cast<float *>(base + res_b + part_b + G_b);
+    ls->y = reinterpret_cast<float *>(base + res_b + part_b + G_b);
     *out = ls;
     return CORE_OK;
 }
@@ -403,9 +410,20 @@ int core_gd_step(core_ctx *ctx, core_ls *ls, float h, float *x_dev) {
     if (int rc = check_ctx(ctx)) return rc;
     if (!ls || !x_dev || ls->d != ctx->d || ls->device != ctx->device) return CORE_EINVAL;
     if (int rc = ls_gradients_into(ctx, ls, x_dev, ls->G)) return rc;
-    if (int rc = core_round(ctx, ls->G, CORE_F32, ls->n, ls->d, ctx->pbar, ls->gt)) return rc;
-    CORE_CUDA(ctx, launch_axpy(x_dev, ls->gt, h, ls->d, ctx->stream));
-    return CORE_OK;
+    // x <- x - h * gtilde inside the reconstruction: the estimate is never stored
+    const ReconstructEpilogue update{x_dev, h, nullptr, nullptr};
+    return round_with_epilogue(ctx, ls->G, CORE_F32, ls->n, ls->d, ctx->pbar, x_dev, &update);
+}
+
+int core_agd_step(core_ctx *ctx, core_ls *ls, float h, float beta, float *x_dev, float *x_prev_dev) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!ls || !x_dev || !x_prev_dev || x_dev == x_prev_dev || ls->d != ctx->d || ls->device != ctx->device)
+        return CORE_EINVAL;
+    CORE_CUDA(ctx, launch_lookahead(x_dev, x_prev_dev, 1.0f - beta, ls->d, ls->y, ctx->stream));
+    if (int rc = ls_gradients_into(ctx, ls, ls->y, ls->G)) return rc;
+    // x_prev <- x and x <- y - h * gtilde(y), both inside the reconstruction
+    const ReconstructEpilogue update{ls->y, h, x_dev, x_prev_dev};
+    return round_with_epilogue(ctx, ls->G, CORE_F32, ls->n, ls->d, ctx->pbar, x_dev, &update);
 }
 
 int core_ls_loss(core_ctx *ctx, core_ls *ls, const float *x_dev, double *loss_dev) {

@@ -42,12 +42,23 @@ cudaError_t launch_finish_project(const float *partial, int chunks, int32_t n, i
 cudaError_t launch_aggregate(const float *P, int32_t n, int32_t m, float *pbar, cudaStream_t stream);
 
 // out[k - k_begin] = gtilde[k] for k in [k_begin, k_end); k_begin must be a multiple of 2048.
+// With an epilogue the estimate is consumed where it is produced and never stored:
+//   out[k] = base[k] - step * gtilde[k]   (the optimiser update of Algorithms 2 and 4)
+// and, if shift_dst is set, shift_dst[k] = shift_src[k] first (x_prev <- x of Algorithm 4).
+// out may alias base and shift_src; all four arrays are indexed like out.
+struct ReconstructEpilogue {
+    const float *base;
+    float step;
+    const float *shift_src;
+    float *shift_dst;
+};
 cudaError_t launch_reconstruct(const RoundKeys &keys, uint32_t t, const float *pbar, int32_t m,
                                int64_t k_begin, int64_t k_end, float *out, int sm_count,
-                               cudaStream_t stream);
+                               cudaStream_t stream, const ReconstructEpilogue *epilogue = nullptr);
 
-// x[k] -= h * g[k]
-cudaError_t launch_axpy(float *x, const float *g, float h, int64_t d, cudaStream_t stream);
+// y[k] = x[k] + gamma * (x[k] - x_prev[k])   (look-ahead point of Algorithm 4)
+cudaError_t launch_lookahead(const float *x, const float *x_prev, float gamma, int64_t d, float *y,
+                             cudaStream_t stream);
 
 cudaError_t launch_debug_philox(const RoundKeys &keys, uint32_t t, uint32_t j, uint64_t q0, int64_t nq,
                                 uint32_t *words, cudaStream_t stream);

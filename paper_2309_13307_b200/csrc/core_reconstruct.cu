@@ -23,9 +23,10 @@ struct ReconstructArgs {
     int64_t k_begin;
     int64_t k_end;
     int m;
-    int vec_ok;       // out + 4*(q - q_begin) is 16-byte aligned
+    int vec_ok;       // out (and the epilogue arrays) + 4*(q - q_begin) are 16-byte aligned
     uint32_t t;
     RoundKeys keys;
+    ReconstructEpilogue epi;   // base == nullptr: store the estimate itself
 };
 
 constexpr int kRecJStep = 2;                      // vectors generated together per loop step
@@ -115,21 +116,39 @@ reconstruct_kernel(const __grid_constant__ ReconstructArgs a) {
             const int64_t off = (int64_t)((qv[u] - q_begin) << 2);        // offset into out
             const int64_t k = (int64_t)(qv[u] << 2);
             if (a.vec_ok && k + 4 <= a.k_end) {
-                *reinterpret_cast<float4 *>(a.out + off) = r;
+                float4 v = r;
+                if (a.epi.base) {
+                    const float4 b = *reinterpret_cast<const float4 *>(a.epi.base + off);
+                    v = make_float4(fmaf(-a.epi.step, r.x, b.x), fmaf(-a.epi.step, r.y, b.y),
+                                    fmaf(-a.epi.step, r.z, b.z), fmaf(-a.epi.step, r.w, b.w));
+                    if (a.epi.shift_dst) {
+                        const float4 s = *reinterpret_cast<const float4 *>(a.epi.shift_src + off);
+                        *reinterpret_cast<float4 *>(a.epi.shift_dst + off) = s;
+                    }
+                }
+                *reinterpret_cast<float4 *>(a.out + off) = v;
             } else {
                 const float vals[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
-                for (int l = 0; l < 4; ++l)
-                    if (k + l < a.k_end) a.out[off + l] = vals[l];
+                for (int l = 0; l < 4; ++l) {
+                    if (k + l >= a.k_end) continue;
+                    float v = vals[l];
+                    if (a.epi.base) {
+                        v = fmaf(-a.epi.step, v, a.epi.base[off + l]);
+                        if (a.epi.shift_dst) a.epi.shift_dst[off + l] = a.epi.shift_src[off + l];
+                    }
+                    a.out[off + l] = v;
+                }
             }
         }
     }
 }
 
-__global__ void axpy_kernel(float *__restrict__ x, const float *__restrict__ g, float h, int64_t d) {
+__global__ void lookahead_kernel(const float *__restrict__ x, const float *__restrict__ x_prev, float gamma, int64_t d,
+                                 float *__restrict__ y) {
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < d; k += stride)
-        x[k] = fmaf(-h, g[k], x[k]);
+        y[k] = fmaf(gamma, x[k] - x_prev[k], x[k]);
 }
 
 struct DebugArgs {
@@ -176,7 +195,7 @@ unsigned grid_for(int64_t items, int threads, int cap) {
 
 cudaError_t launch_reconstruct(const RoundKeys &keys, uint32_t t, const float *pbar, int32_t m,
                                int64_t k_begin, int64_t k_end, float *out, int sm_count,
-                               cudaStream_t stream) {
+                               cudaStream_t stream, const ReconstructEpilogue *epilogue) {
     if (k_end <= k_begin) return cudaSuccess;
     if (k_begin % (4 * kGroupQ) != 0) return cudaErrorInvalidValue;
     ReconstructArgs a{};
@@ -185,7 +204,14 @@ cudaError_t launch_reconstruct(const RoundKeys &keys, uint32_t t, const float *p
     a.k_begin = k_begin;
     a.k_end = k_end;
     a.m = m;
-    a.vec_ok = (reinterpret_cast<uintptr_t>(out) % 16) == 0 ? 1 : 0;
+    uintptr_t align = reinterpret_cast<uintptr_t>(out);
+    if (epilogue && epilogue->base) {
+        a.epi = *epilogue;
+        align |= reinterpret_cast<uintptr_t>(epilogue->base);
+        if (epilogue->shift_dst)
+            align |= reinterpret_cast<uintptr_t>(epilogue->shift_src) | reinterpret_cast<uintptr_t>(epilogue->shift_dst);
+    }
+    a.vec_ok = (align % 16) == 0 ? 1 : 0;
     a.t = t;
     a.keys = keys;
     const int64_t nq = ((k_end + 3) >> 2) - (k_begin >> 2);
@@ -196,8 +222,9 @@ cudaError_t launch_reconstruct(const RoundKeys &keys, uint32_t t, const float *p
     return cudaGetLastError();
 }
 
-cudaError_t launch_axpy(float *x, const float *g, float h, int64_t d, cudaStream_t stream) {
-    axpy_kernel<<<grid_for(d, 256, 148 * 8), 256, 0, stream>>>(x, g, h, d);
+cudaError_t launch_lookahead(const float *x, const float *x_prev, float gamma, int64_t d, float *y,
+                             cudaStream_t stream) {
+    lookahead_kernel<<<grid_for(d, 256, 148 * 8), 256, 0, stream>>>(x, x_prev, gamma, d, y);
     return cudaGetLastError();
 }
 
