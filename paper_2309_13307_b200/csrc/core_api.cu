@@ -35,7 +35,8 @@ struct core_ls {
     int32_t n, rows;
     int64_t d;
     int device;
-    LsPlan plan;
+    LsPlan plan;         // two passes over A (any shape)
+    LsPlan fused_plan;   // one pass over A (d <= 8192, d % 4 == 0); splits == 0 if it does not apply
     float *res;          // n*rows
     float *part;         // n*splits*d
     float *G;            // n*d
@@ -367,8 +368,10 @@ int core_ls_create(core_ls **out, const float *A_dev, const float *b_dev, int32_
         return CORE_ECUDA;
     }
     ls->plan = make_ls_plan(n, rows, d, sm);
+    ls->fused_plan = make_ls_fused_plan(n, rows, d, sm);
+    const int max_splits = ls->plan.splits > ls->fused_plan.splits ? ls->plan.splits : ls->fused_plan.splits;
     const size_t res_b = round_up((size_t)n * rows * sizeof(float), 256);
-    const size_t part_b = round_up((size_t)n * ls->plan.splits * (size_t)d * sizeof(float), 256);
+    const size_t part_b = round_up((size_t)n * max_splits * (size_t)d * sizeof(float), 256);
     const size_t G_b = round_up((size_t)n * (size_t)d * sizeof(float), 256);
     const size_t gt_b = round_up((size_t)d * sizeof(float), 256);
     char *base = nullptr;
@@ -394,6 +397,13 @@ int core_ls_destroy(core_ls *ls) {
 }
 
 static int ls_gradients_into(core_ctx *ctx, core_ls *ls, const float *x_dev, float *G) {
+    if (ls_fused_usable(ls->fused_plan, ls->A, x_dev, ls->part)) {
+        // single pass over A: residual and A^T r per row range, then the fixed-order reduce
+        CORE_CUDA(ctx, launch_ls_fused(ls->fused_plan, ls->A, ls->b, x_dev, ls->n, ls->rows, ls->d, ls->part,
+                                       ctx->stream));
+        CORE_CUDA(ctx, launch_ls_reduce(ls->fused_plan, ls->part, ls->n, ls->rows, ls->d, G, ctx->stream));
+        return CORE_OK;
+    }
     CORE_CUDA(ctx, launch_ls_residual(ls->A, ls->b, x_dev, ls->n, ls->rows, ls->d, ls->res, ctx->stream));
     CORE_CUDA(ctx, launch_ls_at_r(ls->plan, ls->A, ls->res, ls->n, ls->rows, ls->d, ls->part, ctx->stream));
     CORE_CUDA(ctx, launch_ls_reduce(ls->plan, ls->part, ls->n, ls->rows, ls->d, G, ctx->stream));

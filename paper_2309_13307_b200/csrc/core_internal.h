@@ -80,6 +80,13 @@ cudaError_t launch_ls_at_r(const LsPlan &plan, const float *A, const float *res,
                            int64_t d, float *part, cudaStream_t stream);
 cudaError_t launch_ls_reduce(const LsPlan &plan, const float *part, int32_t n, int32_t rows, int64_t d,
                              float *G, cudaStream_t stream);
+// Single pass over A for d <= 8192, d % 4 == 0: part[(i*splits + s)*d + k] as above, with the
+// residual of each row formed on the fly (A is read from HBM once instead of twice).  A plan with
+// splits == 0 means the single-pass kernel does not apply to this shape.
+LsPlan make_ls_fused_plan(int32_t n, int32_t rows, int64_t d, int sm_count);
+bool ls_fused_usable(const LsPlan &fused_plan, const float *A, const float *x, const float *part);
+cudaError_t launch_ls_fused(const LsPlan &plan, const float *A, const float *b, const float *x, int32_t n,
+                            int32_t rows, int64_t d, float *part, cudaStream_t stream);
 // loss[0] = (1/n) sum_i 1/(2 rows) sum_r res_i[r]^2, summed in double in a fixed order
 cudaError_t launch_ls_loss(const float *res, int32_t n, int32_t rows, double *loss, cudaStream_t stream);
 

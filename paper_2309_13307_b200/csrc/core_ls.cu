@@ -121,11 +121,142 @@ ls_loss_kernel(const float *__restrict__ res, int64_t total, double scale, doubl
     if (threadIdx.x == 0) loss[0] = sh[0] * scale;
 }
 
+// ---- single pass over A (rows of up to 8192 columns) -------------------------------------
+// A CTA owns a range of rows of one machine.  Thread t keeps x and its partial gradient for the
+// columns {4(t + 256c) .. +3, c < C4} in registers.  Rows are prefetched with cp.async into a ring in
+// shared memory, every thread copying exactly the 16-byte pieces it will read back itself, so the
+// ring needs no barrier; the only barrier per row is the one of the dot-product reduction.
+// For row r: res = A[r].x - b[r] (fixed-order reduction), then acc += res * A[r] from the same
+// registers.  A is read from HBM once; the partial gradients of the CTAs of a machine are added by
+// ls_reduce_kernel in ascending order.
+constexpr int kRing = 4;   // rows in flight per CTA
+
+__device__ __forceinline__ void ls_cp_async16(void *smem_dst, const void *gmem_src) {
+    const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+
+template <int C4>
+__global__ void __launch_bounds__(kLsThreads, 1)
+ls_fused_kernel(const float *__restrict__ A, const float *__restrict__ b, const float *__restrict__ x, int rows,
+                int d4, int splits, int rows_per_split, float *__restrict__ part) {
+    extern __shared__ __align__(16) unsigned char ls_smem[];
+    float4 *ring = reinterpret_cast<float4 *>(ls_smem);                       // kRing x (C4 * 256) float4
+    float *warp_sums = reinterpret_cast<float *>(ring + kRing * C4 * kLsThreads);   // 2 x 8
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int i = blockIdx.y, s = blockIdx.x;
+    const int r_begin = s * rows_per_split;
+    const int r_end = min(r_begin + rows_per_split, rows);
+    const float4 *Ai = reinterpret_cast<const float4 *>(A) + (int64_t)i * rows * d4;
+    const float *bi = b + (int64_t)i * rows;
+
+    float4 xv[C4], acc[C4];
+#pragma unroll
+    for (int c = 0; c < C4; ++c) {
+        const int col = tid + c * kLsThreads;
+        xv[c] = col < d4 ? __ldg(reinterpret_cast<const float4 *>(x) + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+        acc[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+
+    auto prefetch = [&](int r) {
+        if (r < r_end) {
+            float4 *slot = ring + (size_t)((r - r_begin) % kRing) * C4 * kLsThreads;
+            const float4 *row = Ai + (int64_t)r * d4;
+#pragma unroll
+            for (int c = 0; c < C4; ++c) {
+                const int col = tid + c * kLsThreads;
+                if (col < d4) ls_cp_async16(slot + col, row + col);
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");      // one group per row, empty past the end
+    };
+
+#pragma unroll
+    for (int p = 0; p < kRing - 1; ++p) prefetch(r_begin + p);
+
+    for (int r = r_begin; r < r_end; ++r) {
+        prefetch(r + kRing - 1);
+        asm volatile("cp.async.wait_group %0;" ::"n"(kRing - 1) : "memory");   // row r has landed (own pieces)
+        const float4 *slot = ring + (size_t)((r - r_begin) % kRing) * C4 * kLsThreads;
+        float4 av[C4];
+        float p0 = 0.f, p1 = 0.f, p2 = 0.f, p3 = 0.f;
+#pragma unroll
+        for (int c = 0; c < C4; ++c) {
+            const int col = tid + c * kLsThreads;
+            av[c] = col < d4 ? slot[col] : make_float4(0.f, 0.f, 0.f, 0.f);
+            p0 = fmaf(av[c].x, xv[c].x, p0);
+            p1 = fmaf(av[c].y, xv[c].y, p1);
+            p2 = fmaf(av[c].z, xv[c].z, p2);
+            p3 = fmaf(av[c].w, xv[c].w, p3);
+        }
+        float p = (p0 + p1) + (p2 + p3);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) p += __shfl_xor_sync(0xFFFFFFFFu, p, off);
+        float *sums = warp_sums + ((r - r_begin) & 1) * (kLsThreads / 32);
+        if (lane == 0) sums[warp] = p;
+        __syncthreads();
+        float dot = 0.f;
+#pragma unroll
+        for (int w = 0; w < kLsThreads / 32; ++w) dot += sums[w];
+        const float res = dot - __ldg(bi + r);
+#pragma unroll
+        for (int c = 0; c < C4; ++c) {
+            acc[c].x = fmaf(av[c].x, res, acc[c].x);
+            acc[c].y = fmaf(av[c].y, res, acc[c].y);
+            acc[c].z = fmaf(av[c].z, res, acc[c].z);
+            acc[c].w = fmaf(av[c].w, res, acc[c].w);
+        }
+    }
+    float4 *out = reinterpret_cast<float4 *>(part) + ((int64_t)i * splits + s) * d4;
+#pragma unroll
+    for (int c = 0; c < C4; ++c) {
+        const int col = tid + c * kLsThreads;
+        if (col < d4) out[col] = acc[c];
+    }
+}
+
 bool vec_ok_for(const float *A, int64_t d) {
     return (reinterpret_cast<uintptr_t>(A) % 16) == 0 && d % 4 == 0;
 }
 
 }  // namespace
+
+LsPlan make_ls_fused_plan(int32_t n, int32_t rows, int64_t d, int sm_count) {
+    LsPlan p{};
+    if (d % 4 != 0 || d > 4 * 8 * kLsThreads) return p;     // splits == 0: not available
+    int per_machine = sm_count / n;                          // one CTA per SM, machines side by side
+    if (per_machine < 1) per_machine = 1;
+    if (per_machine > rows) per_machine = rows;
+    p.rows_per_split = (rows + per_machine - 1) / per_machine;
+    p.splits = (rows + p.rows_per_split - 1) / p.rows_per_split;
+    return p;
+}
+
+cudaError_t launch_ls_fused(const LsPlan &plan, const float *A, const float *b, const float *x, int32_t n,
+                            int32_t rows, int64_t d, float *part, cudaStream_t stream) {
+    const int d4 = (int)(d / 4);
+    int c4 = 1;
+    while (c4 * kLsThreads < d4) c4 *= 2;
+    const size_t smem = (size_t)kRing * c4 * kLsThreads * 16 + 2 * (kLsThreads / 32) * sizeof(float);
+    dim3 grid(plan.splits, n);
+    auto go = [&](auto kernel) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kernel<<<grid, kLsThreads, smem, stream>>>(A, b, x, rows, d4, plan.splits, plan.rows_per_split, part);
+        return cudaGetLastError();
+    };
+    switch (c4) {
+        case 1: return go(ls_fused_kernel<1>);
+        case 2: return go(ls_fused_kernel<2>);
+        case 4: return go(ls_fused_kernel<4>);
+        default: return go(ls_fused_kernel<8>);
+    }
+}
+
+bool ls_fused_usable(const LsPlan &fused_plan, const float *A, const float *x, const float *part) {
+    return fused_plan.splits > 0 && ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(x) |
+                                      reinterpret_cast<uintptr_t>(part)) % 16) == 0;
+}
 
 LsPlan make_ls_plan(int32_t n, int32_t rows, int64_t d, int sm_count) {
     LsPlan p{};
