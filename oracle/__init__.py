@@ -82,6 +82,8 @@ def lib() -> ctypes.CDLL:
             L.oracle_gd_step.restype = None
             L.oracle_agd_step.argtypes = [u64, u32, i32, vp, vp, i32, i32, i64, dbl, dbl, vp, vp, vp, ci]
             L.oracle_agd_step.restype = None
+            L.oracle_gd_step_guarded.argtypes = [u64, u32, i32, vp, vp, i32, i32, i64, dbl, vp, vp, vp]
+            L.oracle_gd_step_guarded.restype = ci
             _lib = L
     return _lib
 
@@ -249,3 +251,14 @@ def agd_step(seed: int, t: int, m: int, A, b, h: float, beta: float, x: np.ndarr
     lib().oracle_agd_step(seed, t, m, _ptr(A), _ptr(b), n, rows, d, float(h), float(beta), _ptr(x), _ptr(x_prev),
                           _ptr(work), 1 if exact else 0)
     return x, x_prev
+
+
+def gd_step_guarded(seed: int, t: int, m: int, A, b, h: float, x: np.ndarray, f_x: float):
+    """One Algorithm-3 iteration (caller-fixed step): returns (x_kept, f(x_kept), accepted)."""
+    A, b, n, rows, d = _ls_arrays(A, b)
+    x = np.array(x, dtype=np.float64, copy=True)
+    f = np.array([f_x], dtype=np.float64)
+    work = np.zeros(d + n * d + n * m + m + d, dtype=np.float64)
+    acc = lib().oracle_gd_step_guarded(seed, t, m, _ptr(A), _ptr(b), n, rows, d, float(h), _ptr(x), _ptr(f),
+                                       _ptr(work))
+    return x, float(f[0]), bool(acc)

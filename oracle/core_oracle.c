@@ -242,3 +242,22 @@ void oracle_agd_step(uint64_t seed, uint32_t t, int32_t m, const float *A, const
         x[k] = y[k];
     }
 }
+
+/* ---- Algorithm 3: CORE-GD with the comparison step ---------------------------- */
+
+int oracle_gd_step_guarded(uint64_t seed, uint32_t t, int32_t m, const float *A, const float *b, int32_t n,
+                           int32_t rows, int64_t d, double h, double *x, double *f_x, double *work) {
+    double *trial = work; /* d doubles, then the gd-step work area */
+    double *rest = work + d;
+    for (int64_t k = 0; k < d; ++k) trial[k] = x[k];
+    /* trial point x~ = x - h * gradient estimate at x */
+    oracle_gd_step(seed, t, m, A, b, n, rows, d, h, trial, rest, 0);
+    /* x^{k+1} = argmin over {x^k, x~} of f; a tie keeps x^k */
+    double f_trial = oracle_ls_loss(A, b, n, rows, d, trial);
+    if (f_trial < *f_x) {
+        for (int64_t k = 0; k < d; ++k) x[k] = trial[k];
+        *f_x = f_trial;
+        return 1;
+    }
+    return 0;
+}

@@ -123,6 +123,17 @@ void oracle_agd_step(uint64_t seed, uint32_t t, int32_t m, const float *A, const
                      int32_t rows, int64_t d, double h, double beta, double *x, double *x_prev,
                      double *work, int exact);
 
+/*
+ * One iteration of the non-convex variant (Algorithm 3, "CORE-GD in Non-convex Optimization")
+ * with a step h fixed by the caller (its Option II: h depends only on constants of the problem):
+ * trial x~ = x - h * gtilde(x) with round index t, then x <- argmin over {x, x~} of f, a tie
+ * keeping x.  *f_x holds f(x) on entry and f of the kept point on return.  Returns 1 if the
+ * trial point was accepted.  Option I's step rule is not restated: the statistic it needs is
+ * garbled in the algorithm's text.  work: d doubles more than gd_step needs.
+ */
+int oracle_gd_step_guarded(uint64_t seed, uint32_t t, int32_t m, const float *A, const float *b, int32_t n,
+                           int32_t rows, int64_t d, double h, double *x, double *f_x, double *work);
+
 #ifdef __cplusplus
 }
 #endif
