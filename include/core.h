@@ -198,6 +198,20 @@ int core_gd_step(core_ctx *ctx, core_ls *ls, float h, float *x_dev);
  */
 int core_agd_step(core_ctx *ctx, core_ls *ls, float h, float beta, float *x_dev, float *x_prev_dev);
 
+/*
+ * One iteration of the variant with the comparison step ("CORE-GD in Non-convex
+ * Optimization", Algorithm 3) with a step h fixed by the caller (its Option II, where h
+ * depends only on constants of the problem): trial point x~ = x - h * gtilde(x) from one
+ * round (current t, then t <- t + 1); x <- argmin over {x, x~} of f, a tie keeping x.
+ *   f_dev         one double: f(x) on entry, f of the kept point on return
+ *   accepted_dev  one int32 (may be NULL): 1 if the trial point was taken
+ * The comparison is made on the device; the call does not synchronise.  Option I's
+ * adaptive step is not offered: the statistic it is built on is garbled in the
+ * algorithm's text.
+ */
+int core_gd_step_guarded(core_ctx *ctx, core_ls *ls, float h, float *x_dev, double *f_dev,
+                         int32_t *accepted_dev);
+
 /* loss_dev[0] = f(x) as a double, computed on the device. */
 int core_ls_loss(core_ctx *ctx, core_ls *ls, const float *x_dev, double *loss_dev);
 

@@ -41,6 +41,8 @@ _SIGNATURES = {
     "core_ls_destroy": ([_c.c_void_p], _c.c_int),
     "core_gd_step": ([_c.c_void_p, _c.c_void_p, _c.c_float, _c.c_void_p], _c.c_int),
     "core_agd_step": ([_c.c_void_p, _c.c_void_p, _c.c_float, _c.c_float, _c.c_void_p, _c.c_void_p], _c.c_int),
+    "core_gd_step_guarded": ([_c.c_void_p, _c.c_void_p, _c.c_float, _c.c_void_p, _c.c_void_p, _c.c_void_p],
+                             _c.c_int),
     "core_ls_loss": ([_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p], _c.c_int),
     "core_ls_gradients": ([_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p], _c.c_int),
     "core_debug_philox": ([_c.c_void_p, _c.c_uint32, _c.c_uint64, _c.c_int64, _c.c_void_p], _c.c_int),
@@ -240,6 +242,13 @@ class Core:
         self._check(lib().core_agd_step(self._h, ls._h, float(h), float(beta), _dev(x_dev, torch.float32, self.d),
                                         _dev(x_prev_dev, torch.float32, self.d)), "core_agd_step")
         return x_dev, x_prev_dev
+
+    def core_gd_step_guarded(self, ls: "LeastSquares", h: float, x_dev: torch.Tensor, f_dev: torch.Tensor,
+                             accepted_dev: torch.Tensor | None = None):
+        acc = ctypes.c_void_p(_dev(accepted_dev, torch.int32, 1)) if accepted_dev is not None else None
+        self._check(lib().core_gd_step_guarded(self._h, ls._h, float(h), _dev(x_dev, torch.float32, self.d),
+                                               _dev(f_dev, torch.float64, 1), acc), "core_gd_step_guarded")
+        return x_dev, f_dev
 
     def core_ls_loss(self, ls: "LeastSquares", x_dev: torch.Tensor, loss_dev: torch.Tensor | None = None):
         if loss_dev is None:

@@ -40,7 +40,9 @@ struct core_ls {
     float *res;          // n*rows
     float *part;         // n*splits*d
     float *G;            // n*d
-    float *y;            // d: look-ahead point of the accelerated step
+    float *y;            // d: look-ahead point of the accelerated step / trial point of the guarded step
+    double *f_trial;     // loss at the trial point
+    int *accepted;       // 1 if the last guarded step took the trial point
 };
 
 namespace {
@@ -374,8 +376,9 @@ int core_ls_create(core_ls **out, const float *A_dev, const float *b_dev, int32_
     const size_t part_b = round_up((size_t)n * max_splits * (size_t)d * sizeof(float), 256);
     const size_t G_b = round_up((size_t)n * (size_t)d * sizeof(float), 256);
     const size_t gt_b = round_up((size_t)d * sizeof(float), 256);
+    const size_t scalars_b = 256;                          // trial loss (double) and acceptance flag
     char *base = nullptr;
-    e = cudaMalloc(reinterpret_cast<void **>(&base), res_b + part_b + G_b + gt_b);
+    e = cudaMalloc(reinterpret_cast<void **>(&base), res_b + part_b + G_b + gt_b + scalars_b);
     if (e != cudaSuccess) {
         cudaGetLastError();
         delete ls;
@@ -385,6 +388,8 @@ int core_ls_create(core_ls **out, const float *A_dev, const float *b_dev, int32_
     ls->part = reinterpret_cast<float *>(base + res_b);
     ls->G = reinterpret_cast<float *>(base + res_b + part_b);
     ls->y = reinterpret_cast<float *>(base + res_b + part_b + G_b);
+    ls->f_trial = reinterpret_cast<double *>(base + res_b + part_b + G_b + gt_b);
+    ls->accepted = reinterpret_cast<int *>(base + res_b + part_b + G_b + gt_b + 16);
     *out = ls;
     return CORE_OK;
 }
@@ -434,6 +439,21 @@ int core_agd_step(core_ctx *ctx, core_ls *ls, float h, float beta, float *x_dev,
     // x_prev <- x and x <- y - h * gtilde(y), both inside the reconstruction
     const ReconstructEpilogue update{ls->y, h, x_dev, x_prev_dev};
     return round_with_epilogue(ctx, ls->G, CORE_F32, ls->n, ls->d, ctx->pbar, x_dev, &update);
+}
+
+int core_gd_step_guarded(core_ctx *ctx, core_ls *ls, float h, float *x_dev, double *f_dev, int32_t *accepted_dev) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!ls || !x_dev || !f_dev || ls->d != ctx->d || ls->device != ctx->device) return CORE_EINVAL;
+    if (int rc = ls_gradients_into(ctx, ls, x_dev, ls->G)) return rc;
+    // trial point y = x - h * gtilde, written by the reconstruction; x is left untouched
+    const ReconstructEpilogue trial{x_dev, h, nullptr, nullptr};
+    if (int rc = round_with_epilogue(ctx, ls->G, CORE_F32, ls->n, ls->d, ctx->pbar, ls->y, &trial)) return rc;
+    CORE_CUDA(ctx, launch_ls_residual(ls->A, ls->b, ls->y, ls->n, ls->rows, ls->d, ls->res, ctx->stream));
+    CORE_CUDA(ctx, launch_ls_loss(ls->res, ls->n, ls->rows, ls->f_trial, ctx->stream));
+    // decided on the device: no host synchronisation inside the step
+    CORE_CUDA(ctx, launch_keep_better(ls->f_trial, ls->y, ls->d, f_dev, x_dev, ls->accepted, accepted_dev,
+                                      ctx->stream));
+    return CORE_OK;
 }
 
 int core_ls_loss(core_ctx *ctx, core_ls *ls, const float *x_dev, double *loss_dev) {

@@ -87,6 +87,11 @@ LsPlan make_ls_fused_plan(int32_t n, int32_t rows, int64_t d, int sm_count);
 bool ls_fused_usable(const LsPlan &fused_plan, const float *A, const float *x, const float *part);
 cudaError_t launch_ls_fused(const LsPlan &plan, const float *A, const float *b, const float *x, int32_t n,
                             int32_t rows, int64_t d, float *part, cudaStream_t stream);
+// Comparison step of Algorithm 3, on the device: if *f_trial < *f then x <- trial, *f <- *f_trial and the
+// flag is 1, otherwise nothing changes and the flag is 0 (a tie keeps x).  flag_scratch is a device int
+// owned by the caller of this function; flag_out (may be null) receives a copy.
+cudaError_t launch_keep_better(const double *f_trial, const float *trial, int64_t d, double *f, float *x,
+                               int *flag_scratch, int32_t *flag_out, cudaStream_t stream);
 // loss[0] = (1/n) sum_i 1/(2 rows) sum_r res_i[r]^2, summed in double in a fixed order
 cudaError_t launch_ls_loss(const float *res, int32_t n, int32_t rows, double *loss, cudaStream_t stream);
 

@@ -215,11 +215,36 @@ ls_fused_kernel(const float *__restrict__ A, const float *__restrict__ b, const 
     }
 }
 
+// Comparison step of Algorithm 3: one thread decides, then every thread copies if told to.
+__global__ void keep_better_decide_kernel(const double *__restrict__ f_trial, double *__restrict__ f,
+                                          int *__restrict__ flag, int32_t *__restrict__ flag_out) {
+    const int take = *f_trial < *f ? 1 : 0;     // a tie keeps the current point
+    if (take) *f = *f_trial;
+    *flag = take;
+    if (flag_out) *flag_out = take;
+}
+
+__global__ void keep_better_copy_kernel(const int *__restrict__ flag, const float *__restrict__ trial, int64_t d,
+                                        float *__restrict__ x) {
+    if (*flag == 0) return;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < d; k += stride) x[k] = trial[k];
+}
+
 bool vec_ok_for(const float *A, int64_t d) {
     return (reinterpret_cast<uintptr_t>(A) % 16) == 0 && d % 4 == 0;
 }
 
 }  // namespace
+
+cudaError_t launch_keep_better(const double *f_trial, const float *trial, int64_t d, double *f, float *x,
+                               int *flag_scratch, int32_t *flag_out, cudaStream_t stream) {
+    keep_better_decide_kernel<<<1, 1, 0, stream>>>(f_trial, f, flag_scratch, flag_out);
+    int64_t blocks = (d + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    keep_better_copy_kernel<<<(unsigned)blocks, 256, 0, stream>>>(flag_scratch, trial, d, x);
+    return cudaGetLastError();
+}
 
 LsPlan make_ls_fused_plan(int32_t n, int32_t rows, int64_t d, int sm_count) {
     LsPlan p{};
