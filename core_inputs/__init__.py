@@ -50,14 +50,6 @@ def _gen(seed: int, device) -> torch.Generator:
     return g
 
 
-def _randn_into(out: torch.Tensor, gen: torch.Generator, piece: int = 1 << 26) -> None:
-    """Fill a 1-D fp32 tensor with N(0,1) in bounded pieces (bounded temporaries)."""
-    flat = out.view(-1)
-    for s in range(0, flat.numel(), piece):
-        e = min(s + piece, flat.numel())
-        flat[s:e].normal_(generator=gen)
-
-
 def gradients(n: int, d: int, seed: int = 0, dist: str = "normal", dtype: str = "f32",
               device="cpu", ld: int | None = None) -> torch.Tensor:
     """G[n, d] (a view into an [n, ld] allocation when ld > d), one row per simulated machine.
