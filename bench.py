@@ -76,8 +76,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--d", type=int, default=None, help="override the coordinate count (development)")
     ap.add_argument("--m", type=int, nargs="*", default=None, help="override the m sweep (development)")
-    ap.add_argument("--workload", default="sweep", choices=["sweep", "leastsq"],
-                    help="sweep: the headline CORE round; leastsq: the CORE-GD step (secondary line)")
+    ap.add_argument("--workload", default="sweep", choices=["sweep", "leastsq", "resnet50", "gpt2small", "tiny"],
+                    help="sweep: the headline CORE round; resnet50 / gpt2small / tiny: the round at the other evaluation "
+                         "shapes; leastsq: the CORE-GD step (secondary lines)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     return ap.parse_args()
@@ -169,7 +170,7 @@ def cpu_baseline_sample(budget_s: float = 15.0):
     n_s, m_s = 2, 8
     d_s = 1 << 18
     dt, units = oracle_mini_round(d_s, m_s, n_s, threads)          # calibration
-    scale = max(1, min(64, int(budget_s / max(dt, 1e-3))))
+    scale = max(1, min(1024, int(budget_s / max(dt, 1e-3))))
     if scale > 1:
         d_s *= scale
         dt, units = oracle_mini_round(d_s, m_s, n_s, threads)
@@ -240,7 +241,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     core_mod.lib()                                   # fails loudly if the CUDA library is missing
-    w = core_inputs.WORKLOADS["sweep"]
+    w = core_inputs.WORKLOADS[args.workload]
     d = args.d or w.d
     ms = tuple(args.m) if args.m else w.m
     n = w.n
@@ -371,8 +372,8 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"sweep: d={d} fp32, n={n}, N(0,1) gradients, m in {list(ms)}; one round per m",
-                   "l2": "inputs (8 GB of gradients per replica) are larger than L2; no flush needed",
+        "config": {"workload": f"{w.name}: d={d} {w.dtype}, n={n}, {w.dist} gradients, m in {list(ms)}; one round per m",
+                   "l2": f"inputs ({n * d * G.element_size() / 1e9:.2f} GB of gradients per replica) against a 126 MB L2; no flush",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": 4 * len(ms) * args.steps,
         "roofline": roofline, "sweep": sweep, "cpu_baseline": cpu,

@@ -24,9 +24,17 @@ struct ProjectPlan {
     int grid_y;       // CTAs across vectors
     int64_t tiles;    // ceil(d / (4 * tile_q))
     size_t smem;      // dynamic shared memory per CTA
+    int mma;          // 1: the tensor-core kernel (9..16 machines, m >= 64) runs this pass
 };
 
 ProjectPlan make_project_plan(int32_t n_group, int32_t m, int64_t d, int dtype, int sm_count);
+
+// Tensor-core variant of the projection pass (core_project_mma.cu); same partial-sum layout.
+bool project_mma_applies(int32_t n_group, int32_t m);
+void fill_project_mma_plan(ProjectPlan &plan, int32_t m, int64_t d, int dtype, int sm_count);
+cudaError_t launch_project_mma(const ProjectPlan &plan, const RoundKeys &keys, uint32_t t, const void *G,
+                               int dtype, int32_t n, int64_t ldg, int64_t d, int32_t m, uint64_t q_base,
+                               float *partial, cudaStream_t stream);
 
 // One projection pass over coordinates [0, d) of rows G + i*ldg, i < n <= 16.
 // q_base is the global index of the block holding coordinate 0 of G (non-zero when G

@@ -69,14 +69,21 @@ def test_ragged_sizes(core_mod, d, m, n):
     (17, 5, 20_001, "f32", "normal"),            # more than one machine group
     (3, 600, 9_001, "bf16", "normal"),           # more vectors than one CTA row holds
     (5, 1030, 8_200, "f32", "normal"),
+    (2, 5000, 4_100, "f32", "normal"),           # more vectors than one reconstruction table chunk (2048)
+    (1, 2049, 1_000, "bf16", "normal"),
+    (40, 3, 4_097, "bf16", "student_t3"),        # three machine groups
+    (16, 130, 20_003, "bf16", "student_t3"),     # 9..16 machines and m >= 64: the tensor-core projection
+    (11, 64, 9_001, "f32", "scaled_normal"),
+    (9, 200, 70_000, "f32", "normal"),
+    (25, 72, 3_000, "f32", "normal"),            # two tensor-core passes: 16 machines, then 9
 ])
 def test_medium_sizes(core_mod, n, m, d, dtype, dist):
     G = core_inputs.gradients(n, d, seed=11, dist=dist, dtype=dtype, device="cuda")
     check_round(core_mod, G, m, seed=5, t=1)
 
 
-def test_unaligned_rows_and_leading_dimension(core_mod):
-    n, d, m = 3, 5003, 7
+@pytest.mark.parametrize("n,d,m", [(3, 5003, 7), (10, 3001, 70)])     # scalar and tensor-core projection
+def test_unaligned_rows_and_leading_dimension(core_mod, n, d, m):
     for dtype in ("f32", "bf16"):
         # ld > d with an odd stride, and a base pointer that is not 16-byte aligned
         store = core_inputs.gradients(n, d + 1, seed=2, dtype=dtype, device="cuda", ld=d + 9)
