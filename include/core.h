@@ -95,7 +95,10 @@ int core_last_cuda_error(const core_ctx *ctx);
  *   P_dev   n*m floats, row-major.
  * fp32 multiply-add with two-level fp32 accumulation and a fixed reduction
  * order: results are bitwise reproducible for a given (n, m, d, dtype).
- * n > 16 is processed in groups of 16 machines.  May grow the workspace.
+ * n > 16 is processed in groups of 16 machines.  A group of 9..16 machines
+ * with m >= 64 forms its products on the tensor cores with every operand split
+ * into a tf32 head and tail (same error bar, same reproducibility).  May grow
+ * the workspace.
  */
 int core_project(core_ctx *ctx, const void *G_dev, int dtype, int32_t n, int64_t ldg, float *P_dev);
 
