@@ -82,6 +82,16 @@ size_t core_workspace_bytes(const core_ctx *ctx);
 const char *core_strerror(int code);
 int core_last_cuda_error(const core_ctx *ctx);
 
+/*
+ * Device-side status.  The tensor-memory projection kernel hands buffers between
+ * its warps with barriers whose waits are bounded; a wait that runs out makes
+ * the kernel finish early (its output is then meaningless) and records a
+ * non-zero code in a per-device status word.  This call synchronises the
+ * current device, stores the word in *status_out (host pointer; 0 = every wait
+ * was served) and clears it.  Not part of the paper: run-time diagnostics.
+ */
+int core_device_status(int32_t *status_out);
+
 /* ---- the round ------------------------------------------------------------- */
 
 /*

@@ -6,8 +6,8 @@ The work is done by the CUDA library ``libcore_b200.so`` (C ABI in ``include/cor
 ``binding`` marshals torch tensors into it.  ``python -m paper_2309_13307_b200.build``
 compiles the library in-tree.
 """
-from .binding import (CORE_BF16, CORE_ELIMIT, CORE_F32, Core, CoreError, LeastSquares, core_project_static,
-                      exported_symbols, lib, library_path)
+from .binding import (CORE_BF16, CORE_ELIMIT, CORE_F32, Core, CoreError, LeastSquares, core_device_status,
+                      core_project_static, exported_symbols, lib, library_path)
 
 __all__ = ["Core", "LeastSquares", "CoreError", "CORE_F32", "CORE_BF16", "CORE_ELIMIT", "core_project_static",
-           "lib", "library_path", "exported_symbols"]
+           "core_device_status", "lib", "library_path", "exported_symbols"]

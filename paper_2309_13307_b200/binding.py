@@ -29,6 +29,7 @@ _SIGNATURES = {
     "core_workspace_bytes": ([_c.c_void_p], _c.c_size_t),
     "core_strerror": ([_c.c_int], _c.c_char_p),
     "core_last_cuda_error": ([_c.c_void_p], _c.c_int),
+    "core_device_status": ([_c.POINTER(_c.c_int32)], _c.c_int),
     "core_project": ([_c.c_void_p, _c.c_void_p, _c.c_int, _c.c_int32, _c.c_int64, _c.c_void_p], _c.c_int),
     "core_aggregate": ([_c.c_void_p, _c.c_void_p, _c.c_int32, _c.c_void_p], _c.c_int),
     "core_reconstruct": ([_c.c_void_p, _c.c_void_p, _c.c_void_p], _c.c_int),
@@ -121,6 +122,16 @@ def core_debug_project_plan(n: int, m: int, d: int, dtype: int = CORE_F32, sm_co
         raise CoreError(rc, "core_debug_project_plan")
     keys = ("nb", "jt", "uq", "tile_q", "tj", "tq", "grid_x", "grid_y", "tiles", "smem")
     return dict(zip(keys, (int(v) for v in out)))
+
+
+def core_device_status() -> int:
+    """Synchronises the current device; returns and clears the status word that a kernel raises
+    when one of its bounded waits runs out (0: every wait was served)."""
+    out = ctypes.c_int32(0)
+    rc = lib().core_device_status(ctypes.byref(out))
+    if rc != CORE_OK:
+        raise CoreError(rc, "core_device_status")
+    return int(out.value)
 
 
 def core_project_static(seed: int, t: int, m: int, G_dev: torch.Tensor, P_dev: torch.Tensor,

@@ -209,6 +209,17 @@ const char *core_strerror(int code) {
 
 int core_last_cuda_error(const core_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }
 
+int core_device_status(int32_t *status_out) {
+    if (!status_out) return CORE_EINVAL;
+    int status = 0;
+    if (project_tc_take_status(&status) != cudaSuccess) {
+        cudaGetLastError();
+        return CORE_ECUDA;
+    }
+    *status_out = status;
+    return CORE_OK;
+}
+
 int core_project(core_ctx *ctx, const void *G_dev, int dtype, int32_t n, int64_t ldg, float *P_dev) {
     if (int rc = check_ctx(ctx)) return rc;
     if (!G_dev || !P_dev || n < 1 || ldg < ctx->d || !valid_dtype(dtype)) return CORE_EINVAL;

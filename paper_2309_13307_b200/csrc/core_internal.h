@@ -24,7 +24,7 @@ struct ProjectPlan {
     int grid_y;       // CTAs across vectors
     int64_t tiles;    // ceil(d / (4 * tile_q))
     size_t smem;      // dynamic shared memory per CTA
-    int mma;          // 1: the tensor-core kernel (9..16 machines, m >= 64) runs this pass
+    int mma;          // 0: scalar kernel; 1: warp-level tensor-core kernel; 2: tcgen05 kernel
 };
 
 ProjectPlan make_project_plan(int32_t n_group, int32_t m, int64_t d, int dtype, int sm_count);
@@ -35,6 +35,17 @@ void fill_project_mma_plan(ProjectPlan &plan, int32_t m, int64_t d, int dtype, i
 cudaError_t launch_project_mma(const ProjectPlan &plan, const RoundKeys &keys, uint32_t t, const void *G,
                                int dtype, int32_t n, int64_t ldg, int64_t d, int32_t m, uint64_t q_base,
                                float *partial, cudaStream_t stream);
+
+// tcgen05 variant (core_project_tc.cu): 128 vectors per CTA, accumulators in tensor memory; same
+// partial-sum layout.  q_base must be a multiple of 64 blocks.  Its waits are bounded: a wait that
+// runs out raises a device status word, which project_tc_take_status returns and clears after
+// synchronising the device.
+bool project_tc_applies(int32_t n_group, int32_t m);
+void fill_project_tc_plan(ProjectPlan &plan, int32_t m, int64_t d, int dtype, int sm_count);
+cudaError_t launch_project_tc(const ProjectPlan &plan, const RoundKeys &keys, uint32_t t, const void *G,
+                              int dtype, int32_t n, int64_t ldg, int64_t d, int32_t m, uint64_t q_base,
+                              float *partial, cudaStream_t stream);
+cudaError_t project_tc_take_status(int *status);
 
 // One projection pass over coordinates [0, d) of rows G + i*ldg, i < n <= 16.
 // q_base is the global index of the block holding coordinate 0 of G (non-zero when G

@@ -265,6 +265,10 @@ int ilog2(int x) {
 
 ProjectPlan make_project_plan(int32_t n_group, int32_t m, int64_t d, int dtype, int sm_count) {
     ProjectPlan p{};
+    if (project_tc_applies(n_group, m)) {
+        fill_project_tc_plan(p, m, d, dtype, sm_count);
+        return p;
+    }
     if (project_mma_applies(n_group, m)) {
         fill_project_mma_plan(p, m, d, dtype, sm_count);
         return p;
@@ -301,7 +305,8 @@ ProjectPlan make_project_plan(int32_t n_group, int32_t m, int64_t d, int dtype, 
 cudaError_t launch_project(const ProjectPlan &plan, const RoundKeys &keys, uint32_t t, const void *G,
                            int dtype, int32_t n, int64_t ldg, int64_t d, int32_t m, uint64_t q_base,
                            float *partial, cudaStream_t stream) {
-    if (plan.mma) return launch_project_mma(plan, keys, t, G, dtype, n, ldg, d, m, q_base, partial, stream);
+    if (plan.mma == 2) return launch_project_tc(plan, keys, t, G, dtype, n, ldg, d, m, q_base, partial, stream);
+    if (plan.mma == 1) return launch_project_mma(plan, keys, t, G, dtype, n, ldg, d, m, q_base, partial, stream);
     ProjectArgs a{};
     a.G = G;
     a.ldg = ldg;

@@ -1,0 +1,488 @@
+// Projection with the multiply-adds on the 5th-generation tensor cores (tcgen05 + tensor memory).
+//
+// For many machines the projection P = G Xi^T is a dense contraction whose operand Xi is generated on
+// the fly.  A CTA owns 128 vectors and a range of coordinates.  Eight producer warps generate the
+// Gaussians of one stage (128 vectors x 32 coordinates), split every value into a tf32 head and tail
+// (z = hi + lo, both exact in fp32) and write the two planes to shared memory in the K-major
+// core-matrix layout the tensor core reads; in turn they also stage the machines' gradients for the
+// same 32 coordinates (split the same way when they are fp32; bf16 is exact in tf32).  One lane of a
+// ninth warp issues, per 8 coordinates, tcgen05.mma  D[128 vectors x 16 machines] += A[128 x 8] * B[8 x 16]
+// for the products hi*hi, lo*hi (and hi*lo for fp32 gradients).  D lives in tensor memory, double
+// buffered, with the small products in an accumulator of their own: every 8 stages (256 coordinates)
+// four of the producer warps move both to registers with tcgen05.ld and add them to fp32 running
+// sums.  The tensor core's accumulator loses about half an ulp of the running sum per product, always
+// in the same direction, so its chains are kept short and the large and small terms apart.
+// Stage buffers and accumulators are handed over with mbarriers; every wait is bounded, and a wait
+// that runs out sets a device status word and lets the CTA leave through the normal exit (which
+// releases its tensor memory).  The per-CTA partial sums have the layout of the scalar kernel.
+#include "core_internal.h"
+
+#include <cuda_bf16.h>
+
+namespace core {
+
+namespace {
+
+constexpr int kTcProducerWarps = 8;
+constexpr int kTcThreads = 32 * (kTcProducerWarps + 1);
+constexpr int kTcVectors = 128;                 // M of the instruction = vectors per CTA
+constexpr int kTcN = 16;                        // N of the instruction = machines per pass
+constexpr int kTcStageBlocks = 8;               // coordinate blocks per stage: 32 coordinates = 128 B per row
+constexpr int kTcStages = 3;                    // ring of stage buffers
+constexpr int kTcTileStages = 8;                // stages between two drains of the accumulators
+constexpr int kTcTileBlocks = kTcStageBlocks * kTcTileStages;       // 64 blocks = 256 coordinates
+constexpr uint32_t kTcPlaneA = kTcVectors * 128;                    // bytes of one plane of Xi per stage
+constexpr uint32_t kTcPlaneB = kTcN * 128;                          // bytes of one plane of G per stage
+constexpr uint32_t kTcStageBytes = 2 * kTcPlaneA + 2 * kTcPlaneB;
+constexpr uint32_t kTcBarrierBytes = 128;
+constexpr uint32_t kTcSmemBytes = kTcStages * kTcStageBytes + kTcBarrierBytes + 1024;   // + alignment slack
+constexpr uint32_t kTcTmemColumns = 64;         // two buffers x (head products, tail products) x 16 columns
+constexpr uint32_t kTcSpinLimit = 1u << 22;
+
+__device__ int g_tc_status;                     // 0, or the code of a wait that ran out
+
+struct TcArgs {
+    const void *G;
+    int64_t ldg;
+    int64_t d;
+    int64_t tiles;
+    uint64_t q_base;
+    float *partial;
+    int n;
+    int m;
+    int aligned;
+    uint32_t t;
+    RoundKeys keys;
+};
+
+// ---- thin wrappers over the PTX this kernel needs --------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the phase did not complete within the limit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t spin = 0; spin < kTcSpinLimit; ++spin)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t columns) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(columns) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_free(uint32_t taddr, uint32_t columns) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(columns) : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem], tf32 operands, fp32 accumulate, M = 128, N = 16, K = 8.
+// The descriptors arrive as (low word, high word): only the low word (address field) varies.
+__device__ __forceinline__ void tc_mma_tf32(uint32_t d_tmem, uint32_t a_lo32, uint32_t b_lo32, uint32_t desc_hi32,
+                                            uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo32), "r"(b_lo32), "r"(desc_hi32), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 16 consecutive fp32 columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_load16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int c = 0; c < 16; ++c) v[c] = __uint_as_float(r[c]);
+}
+template <uint32_t OFFSET = 0>
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, float x, float y, float z, float w) {
+    asm volatile("st.shared.v4.f32 [%0+%5], {%1, %2, %3, %4};" ::"r"(addr), "f"(x), "f"(y), "f"(z), "f"(w), "n"(OFFSET)
+                 : "memory");
+}
+
+// Shared-memory matrix descriptor, K-major, no swizzle: a core matrix is 8 rows x 16 bytes stored
+// contiguously (128 B); the two core matrices of one instruction along K are `kLbo` bytes apart, groups
+// of eight rows `kSbo` bytes apart.  Fields: address >> 4 at bit 0, kLbo >> 4 at bit 16, kSbo >> 4 at
+// bit 32, descriptor version 1 at bit 46, layout type 0 (no swizzle) at bit 61.
+constexpr uint32_t kLbo = 128;
+constexpr uint32_t kSbo = 128 * kTcStageBlocks;    // 1024: eight 16-byte chunks per row
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | ((kLbo >> 4) << 16); }
+constexpr uint32_t kDescHi = (kSbo >> 4) | (1u << 14);
+// Byte offset of the 16-byte chunk (row, c) inside a plane.
+__device__ __forceinline__ uint32_t plane_offset(int row, int c) {
+    return (uint32_t)(row >> 3) * kSbo + (uint32_t)c * kLbo + (uint32_t)(row & 7) * 16u;
+}
+// Instruction descriptor: fp32 accumulator (1 at bit 4), tf32 A and B (2 at bits 7 and 10), both K-major,
+// N >> 3 at bit 17, M >> 4 at bit 24.
+constexpr uint32_t kIdesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kTcN >> 3) << 17) |
+                            ((uint32_t)(kTcVectors >> 4) << 24);
+
+__device__ __forceinline__ float tf32_head(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
+
+// Head and tail of the four Gaussians of vector (lane + 32 U) into the two planes of a stage.
+template <int U>
+__device__ __forceinline__ void store_split(uint32_t dst, const float4 &z) {
+    const float hx = tf32_head(z.x), hy = tf32_head(z.y), hz = tf32_head(z.z), hw = tf32_head(z.w);
+    st_shared_v4<U * 4 * kSbo>(dst, hx, hy, hz, hw);
+    st_shared_v4<U * 4 * kSbo + kTcPlaneA>(dst, z.x - hx, z.y - hy, z.z - hz, z.w - hw);
+}
+
+// The same probe as mbar_try_wait, allowed to sleep in hardware for up to about `ns` before it answers.
+__device__ __forceinline__ bool mbar_try_wait_patient(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+
+template <typename GT>
+__global__ void __launch_bounds__(kTcThreads, 2)
+project_tc_kernel(const __grid_constant__ TcArgs a) {
+    constexpr bool BF16 = sizeof(GT) == 2;
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;                    // stage buffers, 1024-byte aligned
+    unsigned char *const smem = smem_raw + (base - raw);
+    const uint32_t bars = base + kTcStages * kTcStageBytes;
+    const uint32_t bar_full = bars, bar_empty = bars + 8 * kTcStages;
+    const uint32_t bar_acc_full = bars + 16 * kTcStages, bar_acc_empty = bar_acc_full + 16, bar_done = bar_acc_full + 32;
+    volatile uint32_t *const words = reinterpret_cast<volatile uint32_t *>(smem + kTcStages * kTcStageBytes + 16 * kTcStages + 40);
+    volatile uint32_t *const tmem_slot = words;                      // written by tcgen05.alloc
+    volatile uint32_t *const abort_flag = words + 1;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const GT *G = static_cast<const GT *>(a.G);
+
+    if (tid == 0) {
+        for (int s = 0; s < kTcStages; ++s) {
+            mbar_init(bar_full + 8 * s, 32 * kTcProducerWarps);      // one arrival per producer thread
+            mbar_init(bar_empty + 8 * s, 1);                         // tcgen05.commit
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_acc_full + 8 * b, 1);                      // tcgen05.commit
+            mbar_init(bar_acc_empty + 8 * b, 4);                     // one arrival per draining warp
+        }
+        mbar_init(bar_done, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == kTcProducerWarps) tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTcTmemColumns);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t taddr = *tmem_slot;
+
+    const int64_t per = (a.tiles + gridDim.x - 1) / gridDim.x;
+    const int64_t tile_begin = (int64_t)blockIdx.x * per;
+    const int64_t tile_end = min(tile_begin + per, a.tiles);
+    auto stages_of = [&](int64_t tile) {
+        const int64_t left = a.d - tile * (4 * kTcTileBlocks);
+        const int64_t st = (left + 4 * kTcStageBlocks - 1) / (4 * kTcStageBlocks);
+        return (int)(st < kTcTileStages ? st : kTcTileStages);
+    };
+    auto give_up = [&](int code) {
+        *abort_flag = 1;
+        atomicMax(&g_tc_status, code);
+    };
+    // Whole-warp wait.  The common case (the phase completed long ago) costs one probe and one vote.
+    auto warp_wait = [&](uint32_t bar, uint32_t parity, int code) {
+        if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+        bool ok = *abort_flag == 0 && mbar_wait(bar, parity);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok && lane == 0) give_up(code);
+        return ok;
+    };
+
+    if (warp < kTcProducerWarps) {
+        // ---- producers: generate, split, store; warps 0..3 also drain the accumulators -------------
+        float outer[kTcN];
+#pragma unroll
+        for (int c = 0; c < kTcN; ++c) outer[c] = 0.f;
+        const int jbase = blockIdx.y * kTcVectors + lane;            // this thread's vectors: jbase + 32 u
+        auto drain = [&](int64_t local_tile) {
+            const uint32_t b = (uint32_t)(local_tile & 1);
+            if (!warp_wait(bar_acc_full + 8 * b, (uint32_t)((local_tile >> 1) & 1), 3)) return;
+            tc_fence_after_sync();
+            float head[16], tail[16];
+            const uint32_t lane_base = taddr + ((uint32_t)(warp * 32) << 16) + b * (2 * kTcN);
+            tmem_load16(lane_base, head);
+            tmem_load16(lane_base + kTcN, tail);
+#pragma unroll
+            for (int c = 0; c < kTcN; ++c) outer[c] += head[c] + tail[c];
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * b);
+        };
+
+        // Gradient staging is shared out among the producer warps in turn: DUTY warps serve a stage, one
+        // 16-byte piece per thread, fetched one stage ahead so that the load is in flight while the
+        // previous stage is generated.
+        constexpr int DUTY = BF16 ? 2 : 4;                          // warps on duty per stage
+        const uint32_t duty_phase = (uint32_t)warp / DUTY;            // serves stages c with c % (8 / DUTY) == duty_phase
+        const int duty_piece = (warp % DUTY) * 32 + lane;             // and always the same piece of them
+        const int duty_i = BF16 ? duty_piece >> 2 : duty_piece >> 3;  // machine
+        const int duty_c = BF16 ? duty_piece & 3 : duty_piece & 7;    // 16-byte piece of the machine's row
+        const GT *const duty_src = G + (int64_t)duty_i * a.ldg + (BF16 ? 8 : 4) * duty_c;
+        uint4 held = make_uint4(0, 0, 0, 0);
+        auto on_duty = [&](uint32_t c) { return (c & (8 / DUTY - 1)) == duty_phase; };
+        auto is_fast = [&](int64_t k0) { return a.aligned && k0 + 4 * kTcStageBlocks <= a.d; };
+        auto fetch = [&](int64_t k0) {
+            if (!is_fast(k0)) return;
+            held = duty_i < a.n ? __ldg(reinterpret_cast<const uint4 *>(duty_src + k0)) : make_uint4(0, 0, 0, 0);
+        };
+        auto put = [&](uint32_t plane_b, int i, int c, float x, float y, float z, float w) {
+            const uint32_t off = plane_b + plane_offset(i, c);
+            if constexpr (BF16) {
+                st_shared_v4(off, x, y, z, w);
+            } else {
+                const float hx = tf32_head(x), hy = tf32_head(y), hz = tf32_head(z), hw = tf32_head(w);
+                st_shared_v4(off, hx, hy, hz, hw);
+                st_shared_v4<kTcPlaneB>(off, x - hx, y - hy, z - hz, w - hw);
+            }
+        };
+        auto deposit = [&](int64_t k0, uint32_t plane_b) {
+            const int i = duty_i, c0 = BF16 ? 2 * duty_c : duty_c;
+            if (is_fast(k0)) {
+                const uint4 h = held;
+                if constexpr (BF16) {
+                    put(plane_b, i, c0, __uint_as_float(h.x << 16), __uint_as_float(h.x & 0xFFFF0000u),
+                        __uint_as_float(h.y << 16), __uint_as_float(h.y & 0xFFFF0000u));
+                    put(plane_b, i, c0 + 1, __uint_as_float(h.z << 16), __uint_as_float(h.z & 0xFFFF0000u),
+                        __uint_as_float(h.w << 16), __uint_as_float(h.w & 0xFFFF0000u));
+                } else {
+                    put(plane_b, i, c0, __uint_as_float(h.x), __uint_as_float(h.y), __uint_as_float(h.z),
+                        __uint_as_float(h.w));
+                }
+                return;
+            }
+            // ragged or unaligned stage: element by element, zero beyond d and beyond n
+            for (int c = c0; c < c0 + (BF16 ? 2 : 1); ++c) {
+                float vals[4] = {0.f, 0.f, 0.f, 0.f};
+                if (i < a.n) {
+#pragma unroll
+                    for (int l = 0; l < 4; ++l) {
+                        const int64_t k = k0 + 4 * c + l;
+                        if (k < a.d) {
+                            if constexpr (BF16)
+                                vals[l] = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short *>(G) +
+                                                                          (int64_t)i * a.ldg + k) << 16);
+                            else
+                                vals[l] = __ldg(reinterpret_cast<const float *>(G) + (int64_t)i * a.ldg + k);
+                        }
+                    }
+                }
+                put(plane_b, i, c, vals[0], vals[1], vals[2], vals[3]);
+            }
+        };
+
+        const uint32_t row_off = plane_offset(lane, warp);           // chunk of vector `lane`; vector lane + 32 u is 4 u row groups on
+        uint32_t s = 0, ph = 0;                                      // ring position and its parity
+        uint32_t count = 0;                                          // stages done (for the staging rota)
+        uint32_t q_hi = (uint32_t)((a.q_base + (uint64_t)tile_begin * kTcTileBlocks) >> 32);
+        JPart jp[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) jp[u] = philox_jpart((uint32_t)(jbase + 32 * u), q_hi, a.keys);
+        const int64_t range_end = min(tile_end * (int64_t)(4 * kTcTileBlocks), a.d);
+        int64_t k0 = tile_begin * (int64_t)(4 * kTcTileBlocks);
+        if (tile_begin < tile_end && on_duty(0)) fetch(k0);
+        bool alive = true;
+        for (int64_t tile = tile_begin; tile < tile_end && alive; ++tile) {
+            const uint64_t q_tile = a.q_base + (uint64_t)tile * kTcTileBlocks;
+            if ((uint32_t)(q_tile >> 32) != q_hi) {                  // once per 2^32 blocks
+                q_hi = (uint32_t)(q_tile >> 32);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) jp[u] = philox_jpart((uint32_t)(jbase + 32 * u), q_hi, a.keys);
+            }
+            const int stages = stages_of(tile);
+            uint32_t q_lo = (uint32_t)q_tile + (uint32_t)warp;
+            for (int st = 0; st < stages; ++st, q_lo += kTcStageBlocks, k0 += 4 * kTcStageBlocks, ++count) {
+                if (!warp_wait(bar_empty + 8 * s, ph ^ 1u, 1)) { alive = false; break; }
+                const uint32_t sb = base + s * kTcStageBytes;
+                if (on_duty(count)) deposit(k0, sb + 2 * kTcPlaneA);
+                else if (on_duty(count + 1) && k0 + 4 * kTcStageBlocks < range_end) fetch(k0 + 4 * kTcStageBlocks);
+                const QPart qp = philox_qpart(q_lo, a.t, a.keys);
+                uint4 w[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) w[u] = philox_combine(jp[u], qp, a.keys);
+                float4 z[4];
+                box_muller4xN<4>(w, z);
+                const uint32_t dst = sb + row_off;
+                store_split<0>(dst, z[0]);
+                store_split<1>(dst, z[1]);
+                store_split<2>(dst, z[2]);
+                store_split<3>(dst, z[3]);
+                fence_proxy_async_smem();                            // my stores, visible to the tensor core
+                mbar_arrive(bar_full + 8 * s);
+                if (++s == kTcStages) { s = 0; ph ^= 1u; }
+            }
+            // the tile before this one has long been multiplied: fold it in while this one is in flight
+            if (alive && warp < 4 && tile > tile_begin) drain(tile - tile_begin - 1);
+        }
+        if (alive && warp < 4 && tile_end > tile_begin) drain(tile_end - tile_begin - 1);
+
+        if (warp < 4) {
+            const int j = blockIdx.y * kTcVectors + warp * 32 + lane;
+            if (j < a.m) {
+#pragma unroll
+                for (int i = 0; i < kTcN; ++i)
+                    if (i < a.n) a.partial[((int64_t)blockIdx.x * a.n + i) * a.m + j] = outer[i];
+            }
+        }
+    } else {
+        // ---- ninth warp: one lane issues the products ------------------------------------------------
+        uint32_t s = 0, ph = 0;
+        bool alive = true;
+        for (int64_t tile = tile_begin; tile < tile_end && alive; ++tile) {
+            const int64_t local = tile - tile_begin;
+            const uint32_t b = (uint32_t)(local & 1);
+            // the accumulators are free once the tile two back has been drained
+            if (!warp_wait(bar_acc_empty + 8 * b, (uint32_t)(((local >> 1) & 1) ^ 1), 4)) break;
+            tc_fence_after_sync();
+            // products with the head of xi and the head of g in one accumulator, the small products
+            // (a tail times a head) in another: the tensor core's accumulation error scales with the
+            // running sum, and the small ones then cost nothing
+            const uint32_t d_head = taddr + b * (2 * kTcN), d_tail = d_head + kTcN;
+            const int stages = stages_of(tile);
+            for (int st = 0; st < stages; ++st) {
+                if (lane == 0) {
+                    bool ok = false;
+                    for (uint32_t spin = 0; spin < kTcSpinLimit && !ok; ++spin)
+                        ok = mbar_try_wait_patient(bar_full + 8 * s, ph, 4000u);
+                    if (ok) {
+                        tc_fence_after_sync();
+                        const uint32_t a_hi = smem_desc_lo(base + s * kTcStageBytes);      // other planes: + bytes >> 4
+                        const uint32_t a_lo = a_hi + (kTcPlaneA >> 4), b_hi = a_hi + (2 * kTcPlaneA >> 4);
+                        const uint32_t b_lo = b_hi + (kTcPlaneB >> 4);
+#pragma unroll
+                        for (int kk = 0; kk < kTcStageBlocks / 2; ++kk) {
+                            const uint32_t step = (uint32_t)kk * 2u * kLbo >> 4;
+                            const uint32_t more = (st | kk) != 0;
+                            tc_mma_tf32(d_head, a_hi + step, b_hi + step, kDescHi, kIdesc, more);
+                            tc_mma_tf32(d_tail, a_lo + step, b_hi + step, kDescHi, kIdesc, more);
+                            if constexpr (!BF16) tc_mma_tf32(d_tail, a_hi + step, b_lo + step, kDescHi, kIdesc, 1u);
+                        }
+                        tc_commit(bar_empty + 8 * s);                 // the stage buffer may be refilled
+                        if (st + 1 == stages) tc_commit(bar_acc_full + 8 * b);
+                    } else {
+                        give_up(5);
+                    }
+                }
+                __syncwarp();
+                if (*abort_flag) { alive = false; break; }
+                if (++s == kTcStages) { s = 0; ph ^= 1u; }
+            }
+        }
+        // nothing of this CTA may still be running on the tensor core when its tensor memory goes back
+        if (lane == 0) {
+            tc_commit(bar_done);
+            if (!mbar_wait(bar_done, 0)) give_up(6);
+        }
+        __syncwarp();
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == kTcProducerWarps) {
+        tc_fence_after_sync();
+        tmem_free(taddr, kTcTmemColumns);
+    }
+}
+
+}  // namespace
+
+bool project_tc_applies(int32_t n_group, int32_t m) {
+    // enough machines for the tensor core to pay, enough vectors to fill most of the 128 rows of the
+    // last CTA row
+    return n_group > 8 && m >= 96 && (m % kTcVectors == 0 || m % kTcVectors >= 64 || m >= 1024);
+}
+
+void fill_project_tc_plan(ProjectPlan &p, int32_t m, int64_t d, int dtype, int sm_count) {
+    (void)dtype;
+    p.mma = 2;
+    p.nb = kTcN;
+    p.jt = 4;
+    p.uq = 1;
+    p.tile_q = kTcTileBlocks;
+    p.tj = 32;                         // producer thread = (lane, warp): 4 vectors x 1 block per stage
+    p.tq = kTcProducerWarps;
+    p.grid_y = (m + kTcVectors - 1) / kTcVectors;
+    p.tiles = (d + 4 * (int64_t)kTcTileBlocks - 1) / (4 * (int64_t)kTcTileBlocks);
+    p.smem = kTcSmemBytes;
+    int64_t gx = (int64_t)sm_count * 2 / p.grid_y;
+    if (gx < 1) gx = 1;
+    if (gx > p.tiles) gx = p.tiles;
+    p.grid_x = (int)gx;
+}
+
+cudaError_t launch_project_tc(const ProjectPlan &plan, const RoundKeys &keys, uint32_t t, const void *G, int dtype,
+                              int32_t n, int64_t ldg, int64_t d, int32_t m, uint64_t q_base, float *partial,
+                              cudaStream_t stream) {
+    if (q_base % kTcTileBlocks != 0 || n > kTcN) return cudaErrorInvalidValue;
+    TcArgs a{};
+    a.G = G;
+    a.ldg = ldg;
+    a.d = d;
+    a.tiles = plan.tiles;
+    a.q_base = q_base;
+    a.partial = partial;
+    a.n = n;
+    a.m = m;
+    const size_t es = dtype == 1 ? 2 : 4;
+    a.aligned = ((reinterpret_cast<uintptr_t>(G) % 16) == 0 && ((size_t)ldg * es) % 16 == 0) ? 1 : 0;
+    a.t = t;
+    a.keys = keys;
+    dim3 grid(plan.grid_x, plan.grid_y);
+    auto go = [&](auto kernel) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem);
+        if (e != cudaSuccess) return e;
+        kernel<<<grid, kTcThreads, plan.smem, stream>>>(a);
+        return cudaGetLastError();
+    };
+    if (dtype == 1) return go(project_tc_kernel<__nv_bfloat16>);
+    return go(project_tc_kernel<float>);
+}
+
+cudaError_t project_tc_take_status(int *status) {
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return e;
+    e = cudaMemcpyFromSymbol(status, g_tc_status, sizeof(int));
+    if (e != cudaSuccess) return e;
+    const int zero = 0;
+    return cudaMemcpyToSymbol(g_tc_status, &zero, sizeof(int));
+}
+
+}  // namespace core
