@@ -252,60 +252,68 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
         // 16-byte piece per thread, fetched one stage ahead so that the load is in flight while the
         // previous stage is generated.
         constexpr int DUTY = BF16 ? 2 : 4;                          // warps on duty per stage
-        const uint32_t duty_phase = (uint32_t)warp / DUTY;            // serves stages c with c % (8 / DUTY) == duty_phase
-        const int duty_piece = (warp % DUTY) * 32 + lane;             // and always the same piece of them
+        constexpr uint32_t ROTA = 8 / DUTY;                           // stages until a warp's turn comes again
+        const uint32_t duty_phase = (uint32_t)warp / DUTY;            // serves stages c with c % ROTA == duty_phase
+        const uint32_t fetch_phase = (duty_phase + ROTA - 1) % ROTA;  // and fetches for them one stage earlier
+        const int duty_piece = (warp % DUTY) * 32 + lane;             // always the same 16-byte piece of the stage
         const int duty_i = BF16 ? duty_piece >> 2 : duty_piece >> 3;  // machine
-        const int duty_c = BF16 ? duty_piece & 3 : duty_piece & 7;    // 16-byte piece of the machine's row
-        const GT *const duty_src = G + (int64_t)duty_i * a.ldg + (BF16 ? 8 : 4) * duty_c;
+        const int duty_c = BF16 ? duty_piece & 3 : duty_piece & 7;    // piece of the machine's row
+        const uint32_t duty_off = 2 * kTcPlaneA + plane_offset(duty_i, BF16 ? 2 * duty_c : duty_c);
+        const int64_t range_begin = tile_begin * (int64_t)(4 * kTcTileBlocks);
+        const int64_t range_end = min(tile_end * (int64_t)(4 * kTcTileBlocks), a.d);
+        // stages of this CTA: the first `fast_stages` lie wholly inside d and can be read 16 bytes at a time
+        const uint32_t total_stages = range_end > range_begin ? (uint32_t)((range_end - range_begin + 31) >> 5) : 0u;
+        const uint32_t fast_stages = a.aligned && range_end > range_begin ? (uint32_t)((range_end - range_begin) >> 5) : 0u;
+        const GT *const duty_src = G + (int64_t)duty_i * a.ldg + range_begin + (BF16 ? 8 : 4) * duty_c;
         uint4 held = make_uint4(0, 0, 0, 0);
-        auto on_duty = [&](uint32_t c) { return (c & (8 / DUTY - 1)) == duty_phase; };
-        auto is_fast = [&](int64_t k0) { return a.aligned && k0 + 4 * kTcStageBlocks <= a.d; };
-        auto fetch = [&](int64_t k0) {
-            if (!is_fast(k0)) return;
-            held = duty_i < a.n ? __ldg(reinterpret_cast<const uint4 *>(duty_src + k0)) : make_uint4(0, 0, 0, 0);
+        auto fetch = [&](uint32_t c) {                                // piece of stage c, if it can be read whole
+            if (c < fast_stages && duty_i < a.n) held = __ldg(reinterpret_cast<const uint4 *>(duty_src + (int64_t)c * 32));
         };
-        auto put = [&](uint32_t plane_b, int i, int c, float x, float y, float z, float w) {
-            const uint32_t off = plane_b + plane_offset(i, c);
+        auto put_slow = [&](uint32_t dst, float x, float y, float z, float w) {
             if constexpr (BF16) {
-                st_shared_v4(off, x, y, z, w);
+                st_shared_v4(dst, x, y, z, w);
             } else {
                 const float hx = tf32_head(x), hy = tf32_head(y), hz = tf32_head(z), hw = tf32_head(w);
-                st_shared_v4(off, hx, hy, hz, hw);
-                st_shared_v4<kTcPlaneB>(off, x - hx, y - hy, z - hz, w - hw);
+                st_shared_v4(dst, hx, hy, hz, hw);
+                st_shared_v4<kTcPlaneB>(dst, x - hx, y - hy, z - hz, w - hw);
             }
         };
-        auto deposit = [&](int64_t k0, uint32_t plane_b) {
-            const int i = duty_i, c0 = BF16 ? 2 * duty_c : duty_c;
-            if (is_fast(k0)) {
-                const uint4 h = held;
+        auto deposit = [&](uint32_t c, uint32_t sb) {                 // stage c into the buffer at sb
+            const uint32_t dst = sb + duty_off;
+            if (c < fast_stages) {
+                const uint4 h = duty_i < a.n ? held : make_uint4(0, 0, 0, 0);
                 if constexpr (BF16) {
-                    put(plane_b, i, c0, __uint_as_float(h.x << 16), __uint_as_float(h.x & 0xFFFF0000u),
-                        __uint_as_float(h.y << 16), __uint_as_float(h.y & 0xFFFF0000u));
-                    put(plane_b, i, c0 + 1, __uint_as_float(h.z << 16), __uint_as_float(h.z & 0xFFFF0000u),
-                        __uint_as_float(h.w << 16), __uint_as_float(h.w & 0xFFFF0000u));
+                    st_shared_v4(dst, __uint_as_float(h.x << 16), __uint_as_float(h.x & 0xFFFF0000u),
+                                 __uint_as_float(h.y << 16), __uint_as_float(h.y & 0xFFFF0000u));
+                    st_shared_v4<kLbo>(dst, __uint_as_float(h.z << 16), __uint_as_float(h.z & 0xFFFF0000u),
+                                       __uint_as_float(h.w << 16), __uint_as_float(h.w & 0xFFFF0000u));
                 } else {
-                    put(plane_b, i, c0, __uint_as_float(h.x), __uint_as_float(h.y), __uint_as_float(h.z),
-                        __uint_as_float(h.w));
+                    const float x = __uint_as_float(h.x), y = __uint_as_float(h.y), z = __uint_as_float(h.z),
+                                w = __uint_as_float(h.w);
+                    const float hx = tf32_head(x), hy = tf32_head(y), hz = tf32_head(z), hw = tf32_head(w);
+                    st_shared_v4(dst, hx, hy, hz, hw);
+                    st_shared_v4<kTcPlaneB>(dst, x - hx, y - hy, z - hz, w - hw);
                 }
                 return;
             }
             // ragged or unaligned stage: element by element, zero beyond d and beyond n
-            for (int c = c0; c < c0 + (BF16 ? 2 : 1); ++c) {
+            const int64_t k0 = range_begin + (int64_t)c * 32 + (BF16 ? 8 : 4) * duty_c;
+            for (int part = 0; part < (BF16 ? 2 : 1); ++part) {
                 float vals[4] = {0.f, 0.f, 0.f, 0.f};
-                if (i < a.n) {
+                if (duty_i < a.n) {
 #pragma unroll
                     for (int l = 0; l < 4; ++l) {
-                        const int64_t k = k0 + 4 * c + l;
+                        const int64_t k = k0 + 4 * part + l;
                         if (k < a.d) {
                             if constexpr (BF16)
                                 vals[l] = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short *>(G) +
-                                                                          (int64_t)i * a.ldg + k) << 16);
+                                                                          (int64_t)duty_i * a.ldg + k) << 16);
                             else
-                                vals[l] = __ldg(reinterpret_cast<const float *>(G) + (int64_t)i * a.ldg + k);
+                                vals[l] = __ldg(reinterpret_cast<const float *>(G) + (int64_t)duty_i * a.ldg + k);
                         }
                     }
                 }
-                put(plane_b, i, c, vals[0], vals[1], vals[2], vals[3]);
+                put_slow(dst + (uint32_t)part * kLbo, vals[0], vals[1], vals[2], vals[3]);
             }
         };
 
@@ -316,9 +324,7 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
         JPart jp[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) jp[u] = philox_jpart((uint32_t)(jbase + 32 * u), q_hi, a.keys);
-        const int64_t range_end = min(tile_end * (int64_t)(4 * kTcTileBlocks), a.d);
-        int64_t k0 = tile_begin * (int64_t)(4 * kTcTileBlocks);
-        if (tile_begin < tile_end && on_duty(0)) fetch(k0);
+        if (duty_phase == 0) fetch(0);
         bool alive = true;
         for (int64_t tile = tile_begin; tile < tile_end && alive; ++tile) {
             const uint64_t q_tile = a.q_base + (uint64_t)tile * kTcTileBlocks;
@@ -329,11 +335,14 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
             }
             const int stages = stages_of(tile);
             uint32_t q_lo = (uint32_t)q_tile + (uint32_t)warp;
-            for (int st = 0; st < stages; ++st, q_lo += kTcStageBlocks, k0 += 4 * kTcStageBlocks, ++count) {
+            for (int st = 0; st < stages; ++st, q_lo += kTcStageBlocks, ++count) {
                 if (!warp_wait(bar_empty + 8 * s, ph ^ 1u, 1)) { alive = false; break; }
                 const uint32_t sb = base + s * kTcStageBytes;
-                if (on_duty(count)) deposit(k0, sb + 2 * kTcPlaneA);
-                else if (on_duty(count + 1) && k0 + 4 * kTcStageBlocks < range_end) fetch(k0 + 4 * kTcStageBlocks);
+                {
+                    const uint32_t turn = count % ROTA;
+                    if (turn == duty_phase) deposit(count, sb);
+                    else if (turn == fetch_phase && count + 1 < total_stages) fetch(count + 1);
+                }
                 const QPart qp = philox_qpart(q_lo, a.t, a.keys);
                 uint4 w[4];
 #pragma unroll
