@@ -1,20 +1,22 @@
 // Projection with the multiply-adds on the 5th-generation tensor cores (tcgen05 + tensor memory).
 //
 // For many machines the projection P = G Xi^T is a dense contraction whose operand Xi is generated on
-// the fly.  A CTA owns 128 vectors and a range of coordinates.  Eight producer warps generate the
-// Gaussians of one stage (128 vectors x 32 coordinates), split every value into a tf32 head and tail
-// (z = hi + lo, both exact in fp32) and write the two planes to shared memory in the K-major
-// core-matrix layout the tensor core reads; in turn they also stage the machines' gradients for the
-// same 32 coordinates (split the same way when they are fp32; bf16 is exact in tf32).  One lane of a
-// ninth warp issues, per 8 coordinates, tcgen05.mma  D[128 vectors x 16 machines] += A[128 x 8] * B[8 x 16]
-// for the products hi*hi, lo*hi (and hi*lo for fp32 gradients).  D lives in tensor memory, double
-// buffered, with the small products in an accumulator of their own: every 8 stages (256 coordinates)
-// four of the producer warps move both to registers with tcgen05.ld and add them to fp32 running
-// sums.  The tensor core's accumulator loses about half an ulp of the running sum per product, always
-// in the same direction, so its chains are kept short and the large and small terms apart.
-// Stage buffers and accumulators are handed over with mbarriers; every wait is bounded, and a wait
-// that runs out sets a device status word and lets the CTA leave through the normal exit (which
-// releases its tensor memory).  The per-CTA partial sums have the layout of the scalar kernel.
+// the fly.  A CTA (8 warps) owns 128 vectors and a range of coordinates.  Per stage (128 vectors x 32
+// coordinates) every thread generates four counters' worth of Gaussians, splits each value into a tf32
+// head and tail (z = hi + lo, both exact in fp32) and writes the two planes to shared memory in the
+// K-major core-matrix layout the tensor core reads; in turn the warps also stage the machines' gradients
+// for the same 32 coordinates (split the same way when they are fp32; bf16 is exact in tf32).  The
+// products of stage c are issued by one lane of warp c % 8 once it has finished generating stage c + 1
+// (and before it reports that stage done, which keeps the issue order equal to the stage order): per 8
+// coordinates  tcgen05.mma  D[128 vectors x 16 machines] += A[128 x 8] * B[8 x 16]  for hi*hi, lo*hi
+// (and hi*lo for fp32 gradients).  D lives in tensor memory, double buffered, with the small products in
+// an accumulator of their own: every 8 stages (256 coordinates) four warps move both to registers with
+// tcgen05.ld and add them to fp32 running sums.  The tensor core's accumulator loses about half an ulp
+// of the running sum per product, always in the same direction, so its chains are kept short and the
+// large and small terms apart.  Stage buffers and accumulators are handed over with mbarriers; every
+// wait is bounded, and a wait that runs out sets a device status word and lets the CTA leave through the
+// normal exit (which releases its tensor memory).  The per-CTA partial sums have the layout of the
+// scalar kernel.
 #include "core_internal.h"
 
 #include <cuda_bf16.h>
@@ -23,8 +25,8 @@ namespace core {
 
 namespace {
 
-constexpr int kTcProducerWarps = 8;
-constexpr int kTcThreads = 32 * (kTcProducerWarps + 1);
+constexpr int kTcWarps = 8;
+constexpr int kTcThreads = 32 * kTcWarps;
 constexpr int kTcVectors = 128;                 // M of the instruction = vectors per CTA
 constexpr int kTcN = 16;                        // N of the instruction = machines per pass
 constexpr int kTcStageBlocks = 8;               // coordinate blocks per stage: 32 coordinates = 128 B per row
@@ -156,6 +158,39 @@ __device__ __forceinline__ void store_split(uint32_t dst, const float4 &z) {
     st_shared_v4<U * 4 * kSbo + kTcPlaneA>(dst, z.x - hx, z.y - hy, z.z - hz, z.w - hw);
 }
 
+// Head and tail of four fp32 gradient values into the two G planes of a stage.
+__device__ __forceinline__ void store_split_b(uint32_t dst, float x, float y, float z, float w) {
+    const float hx = tf32_head(x), hy = tf32_head(y), hz = tf32_head(z), hw = tf32_head(w);
+    st_shared_v4(dst, hx, hy, hz, hw);
+    st_shared_v4<kTcPlaneB>(dst, x - hx, y - hy, z - hz, w - hw);
+}
+
+// One thread's piece of a ragged or unaligned stage (4 coordinates for fp32, 8 for bf16, from k0 on),
+// element by element, zero beyond d and beyond n.  Kept out of line: it is rare.
+template <typename GT>
+__device__ __noinline__ void stage_piece_slowly(const GT *G, int64_t ldg, int64_t d, int n, int i, int64_t k0, uint32_t dst) {
+    constexpr bool BF16 = sizeof(GT) == 2;
+    for (int part = 0; part < (BF16 ? 2 : 1); ++part) {
+        float vals[4] = {0.f, 0.f, 0.f, 0.f};
+        if (i < n) {
+#pragma unroll
+            for (int l = 0; l < 4; ++l) {
+                const int64_t k = k0 + 4 * part + l;
+                if (k < d) {
+                    if constexpr (BF16)
+                        vals[l] = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short *>(G) + (int64_t)i * ldg + k) << 16);
+                    else
+                        vals[l] = __ldg(reinterpret_cast<const float *>(G) + (int64_t)i * ldg + k);
+                }
+            }
+        }
+        if constexpr (BF16)
+            st_shared_v4(dst + (uint32_t)part * kLbo, vals[0], vals[1], vals[2], vals[3]);
+        else
+            store_split_b(dst, vals[0], vals[1], vals[2], vals[3]);
+    }
+}
+
 // The same probe as mbar_try_wait, allowed to sleep in hardware for up to about `ns` before it answers.
 __device__ __forceinline__ bool mbar_try_wait_patient(uint32_t bar, uint32_t parity, uint32_t ns) {
     uint32_t ok;
@@ -189,18 +224,18 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
 
     if (tid == 0) {
         for (int s = 0; s < kTcStages; ++s) {
-            mbar_init(bar_full + 8 * s, 32 * kTcProducerWarps);      // one arrival per producer thread
-            mbar_init(bar_empty + 8 * s, 1);                         // tcgen05.commit
+            mbar_init(bar_full + 8 * s, kTcThreads);                 // one arrival per thread
+            mbar_init(bar_empty + 8 * s, 1);                         // tcgen05.commit of the stage's products
         }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(bar_acc_full + 8 * b, 1);                      // tcgen05.commit
+            mbar_init(bar_acc_full + 8 * b, kTcTileStages);          // one tcgen05.commit per stage of the tile
             mbar_init(bar_acc_empty + 8 * b, 4);                     // one arrival per draining warp
         }
-        mbar_init(bar_done, 1);
+        mbar_init(bar_done, kTcWarps);                               // one tcgen05.commit per warp at the end
         *abort_flag = 0;
         fence_barrier_init();
     }
-    if (warp == kTcProducerWarps) tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTcTmemColumns);
+    if (warp == 0) tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTcTmemColumns);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -226,206 +261,182 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
         if (!ok && lane == 0) give_up(code);
         return ok;
     };
+    // One lane waits, patiently (the hardware may park it between probes).
+    auto lane_wait = [&](uint32_t bar, uint32_t parity, int code) {
+        bool ok = false;
+        for (uint32_t spin = 0; spin < kTcSpinLimit && !ok; ++spin) ok = mbar_try_wait_patient(bar, parity, 2000u);
+        if (!ok) give_up(code);
+        return ok;
+    };
 
-    if (warp < kTcProducerWarps) {
-        // ---- producers: generate, split, store; warps 0..3 also drain the accumulators -------------
-        float outer[kTcN];
+    float outer[kTcN];
 #pragma unroll
-        for (int c = 0; c < kTcN; ++c) outer[c] = 0.f;
-        const int jbase = blockIdx.y * kTcVectors + lane;            // this thread's vectors: jbase + 32 u
-        auto drain = [&](int64_t local_tile) {
-            const uint32_t b = (uint32_t)(local_tile & 1);
-            if (!warp_wait(bar_acc_full + 8 * b, (uint32_t)((local_tile >> 1) & 1), 3)) return;
-            tc_fence_after_sync();
-            float head[16], tail[16];
-            const uint32_t lane_base = taddr + ((uint32_t)(warp * 32) << 16) + b * (2 * kTcN);
-            tmem_load16(lane_base, head);
-            tmem_load16(lane_base + kTcN, tail);
+    for (int c = 0; c < kTcN; ++c) outer[c] = 0.f;
+    const int jbase = blockIdx.y * kTcVectors + lane;                // this thread's vectors: jbase + 32 u
+    auto drain = [&](int64_t local_tile) {                           // warps 0..3: tensor memory -> running sums
+        const uint32_t b = (uint32_t)(local_tile & 1);
+        if (!warp_wait(bar_acc_full + 8 * b, (uint32_t)((local_tile >> 1) & 1), 3)) return;
+        tc_fence_after_sync();
+        float head[16], tail[16];
+        const uint32_t lane_base = taddr + ((uint32_t)(warp * 32) << 16) + b * (2 * kTcN);
+        tmem_load16(lane_base, head);
+        tmem_load16(lane_base + kTcN, tail);
 #pragma unroll
-            for (int c = 0; c < kTcN; ++c) outer[c] += head[c] + tail[c];
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * b);
-        };
+        for (int c = 0; c < kTcN; ++c) outer[c] += head[c] + tail[c];
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_acc_empty + 8 * b);
+    };
 
-        // Gradient staging is shared out among the producer warps in turn: DUTY warps serve a stage, one
-        // 16-byte piece per thread, fetched one stage ahead so that the load is in flight while the
-        // previous stage is generated.
-        constexpr int DUTY = BF16 ? 2 : 4;                          // warps on duty per stage
-        constexpr uint32_t ROTA = 8 / DUTY;                           // stages until a warp's turn comes again
-        const uint32_t duty_phase = (uint32_t)warp / DUTY;            // serves stages c with c % ROTA == duty_phase
-        const uint32_t fetch_phase = (duty_phase + ROTA - 1) % ROTA;  // and fetches for them one stage earlier
-        const int duty_piece = (warp % DUTY) * 32 + lane;             // always the same 16-byte piece of the stage
-        const int duty_i = BF16 ? duty_piece >> 2 : duty_piece >> 3;  // machine
-        const int duty_c = BF16 ? duty_piece & 3 : duty_piece & 7;    // piece of the machine's row
-        const uint32_t duty_off = 2 * kTcPlaneA + plane_offset(duty_i, BF16 ? 2 * duty_c : duty_c);
-        const int64_t range_begin = tile_begin * (int64_t)(4 * kTcTileBlocks);
-        const int64_t range_end = min(tile_end * (int64_t)(4 * kTcTileBlocks), a.d);
-        // stages of this CTA: the first `fast_stages` lie wholly inside d and can be read 16 bytes at a time
-        const uint32_t total_stages = range_end > range_begin ? (uint32_t)((range_end - range_begin + 31) >> 5) : 0u;
-        const uint32_t fast_stages = a.aligned && range_end > range_begin ? (uint32_t)((range_end - range_begin) >> 5) : 0u;
-        const GT *const duty_src = G + (int64_t)duty_i * a.ldg + range_begin + (BF16 ? 8 : 4) * duty_c;
-        uint4 held = make_uint4(0, 0, 0, 0);
-        auto fetch = [&](uint32_t c) {                                // piece of stage c, if it can be read whole
-            if (c < fast_stages && duty_i < a.n) held = __ldg(reinterpret_cast<const uint4 *>(duty_src + (int64_t)c * 32));
-        };
-        auto put_slow = [&](uint32_t dst, float x, float y, float z, float w) {
+    // Gradient staging is shared out among the warps in turn: DUTY warps serve a stage, one 16-byte piece
+    // per thread, fetched one stage ahead so that the load is in flight while the previous stage is
+    // generated.
+    constexpr int DUTY = BF16 ? 2 : 4;                              // warps on duty per stage
+    constexpr uint32_t ROTA = kTcWarps / DUTY;                        // stages until a warp's turn comes again
+    const uint32_t duty_phase = (uint32_t)warp / DUTY;                // serves stages c with c % ROTA == duty_phase
+    const uint32_t fetch_phase = (duty_phase + ROTA - 1) % ROTA;      // and fetches for them one stage earlier
+    const int duty_piece = (warp % DUTY) * 32 + lane;                 // always the same 16-byte piece of the stage
+    const int duty_i = BF16 ? duty_piece >> 2 : duty_piece >> 3;      // machine
+    const int duty_c = BF16 ? duty_piece & 3 : duty_piece & 7;        // piece of the machine's row
+    const uint32_t duty_off = 2 * kTcPlaneA + plane_offset(duty_i, BF16 ? 2 * duty_c : duty_c);
+    const int64_t range_begin = tile_begin * (int64_t)(4 * kTcTileBlocks);
+    const int64_t range_end = min(tile_end * (int64_t)(4 * kTcTileBlocks), a.d);
+    // stages of this CTA: the first `fast_stages` lie wholly inside d and can be read 16 bytes at a time
+    const uint32_t total_stages = range_end > range_begin ? (uint32_t)((range_end - range_begin + 31) >> 5) : 0u;
+    const uint32_t fast_stages = a.aligned && range_end > range_begin ? (uint32_t)((range_end - range_begin) >> 5) : 0u;
+    const GT *const duty_src = G + (int64_t)duty_i * a.ldg + range_begin + (BF16 ? 8 : 4) * duty_c;
+    uint4 held = make_uint4(0, 0, 0, 0);
+    auto fetch = [&](uint32_t c) {                                    // piece of stage c, if it can be read whole
+        if (c < fast_stages && duty_i < a.n) held = __ldg(reinterpret_cast<const uint4 *>(duty_src + (int64_t)c * 32));
+    };
+    auto deposit = [&](uint32_t c, uint32_t sb) {                     // stage c into the buffer at sb
+        const uint32_t dst = sb + duty_off;
+        if (c < fast_stages) {
+            const uint4 h = duty_i < a.n ? held : make_uint4(0, 0, 0, 0);
             if constexpr (BF16) {
-                st_shared_v4(dst, x, y, z, w);
+                st_shared_v4(dst, __uint_as_float(h.x << 16), __uint_as_float(h.x & 0xFFFF0000u),
+                             __uint_as_float(h.y << 16), __uint_as_float(h.y & 0xFFFF0000u));
+                st_shared_v4<kLbo>(dst, __uint_as_float(h.z << 16), __uint_as_float(h.z & 0xFFFF0000u),
+                                   __uint_as_float(h.w << 16), __uint_as_float(h.w & 0xFFFF0000u));
             } else {
-                const float hx = tf32_head(x), hy = tf32_head(y), hz = tf32_head(z), hw = tf32_head(w);
-                st_shared_v4(dst, hx, hy, hz, hw);
-                st_shared_v4<kTcPlaneB>(dst, x - hx, y - hy, z - hz, w - hw);
+                store_split_b(dst, __uint_as_float(h.x), __uint_as_float(h.y), __uint_as_float(h.z), __uint_as_float(h.w));
             }
-        };
-        auto deposit = [&](uint32_t c, uint32_t sb) {                 // stage c into the buffer at sb
-            const uint32_t dst = sb + duty_off;
-            if (c < fast_stages) {
-                const uint4 h = duty_i < a.n ? held : make_uint4(0, 0, 0, 0);
-                if constexpr (BF16) {
-                    st_shared_v4(dst, __uint_as_float(h.x << 16), __uint_as_float(h.x & 0xFFFF0000u),
-                                 __uint_as_float(h.y << 16), __uint_as_float(h.y & 0xFFFF0000u));
-                    st_shared_v4<kLbo>(dst, __uint_as_float(h.z << 16), __uint_as_float(h.z & 0xFFFF0000u),
-                                       __uint_as_float(h.w << 16), __uint_as_float(h.w & 0xFFFF0000u));
-                } else {
-                    const float x = __uint_as_float(h.x), y = __uint_as_float(h.y), z = __uint_as_float(h.z),
-                                w = __uint_as_float(h.w);
-                    const float hx = tf32_head(x), hy = tf32_head(y), hz = tf32_head(z), hw = tf32_head(w);
-                    st_shared_v4(dst, hx, hy, hz, hw);
-                    st_shared_v4<kTcPlaneB>(dst, x - hx, y - hy, z - hz, w - hw);
-                }
-                return;
-            }
-            // ragged or unaligned stage: element by element, zero beyond d and beyond n
-            const int64_t k0 = range_begin + (int64_t)c * 32 + (BF16 ? 8 : 4) * duty_c;
-            for (int part = 0; part < (BF16 ? 2 : 1); ++part) {
-                float vals[4] = {0.f, 0.f, 0.f, 0.f};
-                if (duty_i < a.n) {
-#pragma unroll
-                    for (int l = 0; l < 4; ++l) {
-                        const int64_t k = k0 + 4 * part + l;
-                        if (k < a.d) {
-                            if constexpr (BF16)
-                                vals[l] = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short *>(G) +
-                                                                          (int64_t)duty_i * a.ldg + k) << 16);
-                            else
-                                vals[l] = __ldg(reinterpret_cast<const float *>(G) + (int64_t)duty_i * a.ldg + k);
-                        }
-                    }
-                }
-                put_slow(dst + (uint32_t)part * kLbo, vals[0], vals[1], vals[2], vals[3]);
-            }
-        };
+            return;
+        }
+        stage_piece_slowly<GT>(G, a.ldg, a.d, a.n, duty_i, range_begin + (int64_t)c * 32 + (BF16 ? 8 : 4) * duty_c, dst);
+    };
 
-        const uint32_t row_off = plane_offset(lane, warp);           // chunk of vector `lane`; vector lane + 32 u is 4 u row groups on
-        uint32_t s = 0, ph = 0;                                      // ring position and its parity
-        uint32_t count = 0;                                          // stages done (for the staging rota)
-        uint32_t q_hi = (uint32_t)((a.q_base + (uint64_t)tile_begin * kTcTileBlocks) >> 32);
-        JPart jp[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) jp[u] = philox_jpart((uint32_t)(jbase + 32 * u), q_hi, a.keys);
-        if (duty_phase == 0) fetch(0);
-        bool alive = true;
-        for (int64_t tile = tile_begin; tile < tile_end && alive; ++tile) {
-            const uint64_t q_tile = a.q_base + (uint64_t)tile * kTcTileBlocks;
-            if ((uint32_t)(q_tile >> 32) != q_hi) {                  // once per 2^32 blocks
-                q_hi = (uint32_t)(q_tile >> 32);
-#pragma unroll
-                for (int u = 0; u < 4; ++u) jp[u] = philox_jpart((uint32_t)(jbase + 32 * u), q_hi, a.keys);
-            }
-            const int stages = stages_of(tile);
-            uint32_t q_lo = (uint32_t)q_tile + (uint32_t)warp;
-            for (int st = 0; st < stages; ++st, q_lo += kTcStageBlocks, ++count) {
-                if (!warp_wait(bar_empty + 8 * s, ph ^ 1u, 1)) { alive = false; break; }
-                const uint32_t sb = base + s * kTcStageBytes;
-                {
-                    const uint32_t turn = count % ROTA;
-                    if (turn == duty_phase) deposit(count, sb);
-                    else if (turn == fetch_phase && count + 1 < total_stages) fetch(count + 1);
-                }
-                const QPart qp = philox_qpart(q_lo, a.t, a.keys);
-                uint4 w[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) w[u] = philox_combine(jp[u], qp, a.keys);
-                float4 z[4];
-                box_muller4xN<4>(w, z);
-                const uint32_t dst = sb + row_off;
-                store_split<0>(dst, z[0]);
-                store_split<1>(dst, z[1]);
-                store_split<2>(dst, z[2]);
-                store_split<3>(dst, z[3]);
-                fence_proxy_async_smem();                            // my stores, visible to the tensor core
-                mbar_arrive(bar_full + 8 * s);
-                if (++s == kTcStages) { s = 0; ph ^= 1u; }
-            }
-            // the tile before this one has long been multiplied: fold it in while this one is in flight
-            if (alive && warp < 4 && tile > tile_begin) drain(tile - tile_begin - 1);
-        }
-        if (alive && warp < 4 && tile_end > tile_begin) drain(tile_end - tile_begin - 1);
-
-        if (warp < 4) {
-            const int j = blockIdx.y * kTcVectors + warp * 32 + lane;
-            if (j < a.m) {
-#pragma unroll
-                for (int i = 0; i < kTcN; ++i)
-                    if (i < a.n) a.partial[((int64_t)blockIdx.x * a.n + i) * a.m + j] = outer[i];
-            }
-        }
-    } else {
-        // ---- ninth warp: one lane issues the products ------------------------------------------------
-        uint32_t s = 0, ph = 0;
-        bool alive = true;
-        for (int64_t tile = tile_begin; tile < tile_end && alive; ++tile) {
-            const int64_t local = tile - tile_begin;
-            const uint32_t b = (uint32_t)(local & 1);
-            // the accumulators are free once the tile two back has been drained
-            if (!warp_wait(bar_acc_empty + 8 * b, (uint32_t)(((local >> 1) & 1) ^ 1), 4)) break;
-            tc_fence_after_sync();
-            // products with the head of xi and the head of g in one accumulator, the small products
-            // (a tail times a head) in another: the tensor core's accumulation error scales with the
-            // running sum, and the small ones then cost nothing
-            const uint32_t d_head = taddr + b * (2 * kTcN), d_tail = d_head + kTcN;
-            const int stages = stages_of(tile);
-            for (int st = 0; st < stages; ++st) {
-                if (lane == 0) {
-                    bool ok = false;
-                    for (uint32_t spin = 0; spin < kTcSpinLimit && !ok; ++spin)
-                        ok = mbar_try_wait_patient(bar_full + 8 * s, ph, 4000u);
-                    if (ok) {
-                        tc_fence_after_sync();
-                        const uint32_t a_hi = smem_desc_lo(base + s * kTcStageBytes);      // other planes: + bytes >> 4
-                        const uint32_t a_lo = a_hi + (kTcPlaneA >> 4), b_hi = a_hi + (2 * kTcPlaneA >> 4);
-                        const uint32_t b_lo = b_hi + (kTcPlaneB >> 4);
-#pragma unroll
-                        for (int kk = 0; kk < kTcStageBlocks / 2; ++kk) {
-                            const uint32_t step = (uint32_t)kk * 2u * kLbo >> 4;
-                            const uint32_t more = (st | kk) != 0;
-                            tc_mma_tf32(d_head, a_hi + step, b_hi + step, kDescHi, kIdesc, more);
-                            tc_mma_tf32(d_tail, a_lo + step, b_hi + step, kDescHi, kIdesc, more);
-                            if constexpr (!BF16) tc_mma_tf32(d_tail, a_hi + step, b_lo + step, kDescHi, kIdesc, 1u);
-                        }
-                        tc_commit(bar_empty + 8 * s);                 // the stage buffer may be refilled
-                        if (st + 1 == stages) tc_commit(bar_acc_full + 8 * b);
-                    } else {
-                        give_up(5);
-                    }
-                }
-                __syncwarp();
-                if (*abort_flag) { alive = false; break; }
-                if (++s == kTcStages) { s = 0; ph ^= 1u; }
-            }
-        }
-        // nothing of this CTA may still be running on the tensor core when its tensor memory goes back
+    // Products of one finished stage, issued by one lane.  `st` is the stage's index in its tile of
+    // `stages`, `local` the tile's index in this CTA, (slot, parity) its ring position.
+    auto issue = [&](uint32_t slot, uint32_t parity, int st, int stages, int64_t local) {
         if (lane == 0) {
-            tc_commit(bar_done);
-            if (!mbar_wait(bar_done, 0)) give_up(6);
+            const uint32_t b = (uint32_t)(local & 1);
+            bool ok = true;
+            // the accumulators are free once the tile two back has been drained
+            if (st == 0) ok = lane_wait(bar_acc_empty + 8 * b, (uint32_t)(((local >> 1) & 1) ^ 1), 4);
+            if (ok) ok = lane_wait(bar_full + 8 * slot, parity, 5);
+            if (ok) {
+                tc_fence_after_sync();
+                // products with the head of xi and the head of g in one accumulator, the small products
+                // (a tail times a head) in another: the tensor core's accumulation error scales with the
+                // running sum, and the small ones then cost nothing
+                const uint32_t d_head = taddr + b * (2 * kTcN), d_tail = d_head + kTcN;
+                const uint32_t a_hi = smem_desc_lo(base + slot * kTcStageBytes);          // other planes: + bytes >> 4
+                const uint32_t a_lo = a_hi + (kTcPlaneA >> 4), b_hi = a_hi + (2 * kTcPlaneA >> 4);
+                const uint32_t b_lo = b_hi + (kTcPlaneB >> 4);
+#pragma unroll
+                for (int kk = 0; kk < kTcStageBlocks / 2; ++kk) {
+                    const uint32_t step = (uint32_t)kk * 2u * kLbo >> 4;
+                    const uint32_t more = (st | kk) != 0;
+                    tc_mma_tf32(d_head, a_hi + step, b_hi + step, kDescHi, kIdesc, more);
+                    tc_mma_tf32(d_tail, a_lo + step, b_hi + step, kDescHi, kIdesc, more);
+                    if constexpr (!BF16) tc_mma_tf32(d_tail, a_hi + step, b_lo + step, kDescHi, kIdesc, 1u);
+                }
+                tc_commit(bar_empty + 8 * slot);                      // the stage buffer may be refilled
+                tc_commit(bar_acc_full + 8 * b);                      // one of the tile's kTcTileStages arrivals
+                if (st + 1 == stages)                                 // a short last tile: make up the count
+                    for (int r = stages; r < kTcTileStages; ++r) tc_commit(bar_acc_full + 8 * b);
+                tc_fence_before_sync();                               // issued before this warp's arrival below
+            }
         }
         __syncwarp();
+    };
+
+    const uint32_t row_off = plane_offset(lane, warp);               // chunk of vector `lane`; vector lane + 32 u is 4 u row groups on
+    uint32_t s = 0, ph = 0;                                          // ring position and its parity
+    uint32_t count = 0;                                              // stages done
+    // the stage before the current one, whose products are issued by warp (count - 1) % 8
+    uint32_t prev_s = 0, prev_ph = 0;
+    int prev_st = 0, prev_stages = 0;
+    int64_t prev_local = 0;
+    uint32_t q_hi = (uint32_t)((a.q_base + (uint64_t)tile_begin * kTcTileBlocks) >> 32);
+    JPart jp[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) jp[u] = philox_jpart((uint32_t)(jbase + 32 * u), q_hi, a.keys);
+    if (duty_phase == 0) fetch(0);
+    bool alive = true;
+    for (int64_t tile = tile_begin; tile < tile_end && alive; ++tile) {
+        const uint64_t q_tile = a.q_base + (uint64_t)tile * kTcTileBlocks;
+        if ((uint32_t)(q_tile >> 32) != q_hi) {                      // once per 2^32 blocks
+            q_hi = (uint32_t)(q_tile >> 32);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) jp[u] = philox_jpart((uint32_t)(jbase + 32 * u), q_hi, a.keys);
+        }
+        const int stages = stages_of(tile);
+        uint32_t q_lo = (uint32_t)q_tile + (uint32_t)warp;
+        for (int st = 0; st < stages; ++st, q_lo += kTcStageBlocks, ++count) {
+            if (!warp_wait(bar_empty + 8 * s, ph ^ 1u, 1)) { alive = false; break; }
+            const uint32_t sb = base + s * kTcStageBytes;
+            {
+                const uint32_t turn = count % ROTA;
+                if (turn == duty_phase) deposit(count, sb);
+                else if (turn == fetch_phase && count + 1 < total_stages) fetch(count + 1);
+            }
+            const QPart qp = philox_qpart(q_lo, a.t, a.keys);
+            uint4 w[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) w[u] = philox_combine(jp[u], qp, a.keys);
+            float4 z[4];
+            box_muller4xN<4>(w, z);
+            const uint32_t dst = sb + row_off;
+            store_split<0>(dst, z[0]);
+            store_split<1>(dst, z[1]);
+            store_split<2>(dst, z[2]);
+            store_split<3>(dst, z[3]);
+            // The previous stage's products go out before this warp reports the current stage done, so
+            // that no other warp can be issuing a later stage first.
+            if (count > 0 && (uint32_t)warp == ((count - 1) & (kTcWarps - 1))) {
+                issue(prev_s, prev_ph, prev_st, prev_stages, prev_local);
+                if (*abort_flag) { alive = false; break; }
+            }
+            fence_proxy_async_smem();                                // my stores, visible to the tensor core
+            mbar_arrive(bar_full + 8 * s);
+            prev_s = s; prev_ph = ph; prev_st = st; prev_stages = stages; prev_local = tile - tile_begin;
+            if (++s == kTcStages) { s = 0; ph ^= 1u; }
+        }
+        // the tile before this one has long been multiplied: fold it in while this one is in flight
+        if (alive && warp < 4 && tile > tile_begin) drain(tile - tile_begin - 1);
+    }
+    if (alive && count > 0 && (uint32_t)warp == ((count - 1) & (kTcWarps - 1)))
+        issue(prev_s, prev_ph, prev_st, prev_stages, prev_local);
+    if (alive && warp < 4 && tile_end > tile_begin) drain(tile_end - tile_begin - 1);
+
+    if (warp < 4) {
+        const int j = blockIdx.y * kTcVectors + warp * 32 + lane;
+        if (j < a.m) {
+#pragma unroll
+            for (int i = 0; i < kTcN; ++i)
+                if (i < a.n) a.partial[((int64_t)blockIdx.x * a.n + i) * a.m + j] = outer[i];
+        }
     }
 
+    // nothing of this CTA may still be running on the tensor core when its tensor memory goes back
+    if (lane == 0) tc_commit(bar_done);
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == kTcProducerWarps) {
+    if (warp == 0) {
+        if (lane == 0 && !mbar_wait(bar_done, 0)) give_up(6);
+        __syncwarp();
         tc_fence_after_sync();
         tmem_free(taddr, kTcTmemColumns);
     }
@@ -447,7 +458,7 @@ void fill_project_tc_plan(ProjectPlan &p, int32_t m, int64_t d, int dtype, int s
     p.uq = 1;
     p.tile_q = kTcTileBlocks;
     p.tj = 32;                         // producer thread = (lane, warp): 4 vectors x 1 block per stage
-    p.tq = kTcProducerWarps;
+    p.tq = kTcWarps;
     p.grid_y = (m + kTcVectors - 1) / kTcVectors;
     p.tiles = (d + 4 * (int64_t)kTcTileBlocks - 1) / (4 * (int64_t)kTcTileBlocks);
     p.smem = kTcSmemBytes;

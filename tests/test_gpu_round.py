@@ -42,6 +42,7 @@ def check_round(core_mod, G: torch.Tensor, m: int, seed: int = 1, t: int = 0):
     pbar2, gt2 = ctx.core_round(G)
     assert ctx.core_get_round() == t + 1
     assert torch.equal(pbar2, pbar) and torch.equal(gt2, gt)
+    assert core_mod.core_device_status() == 0        # no bounded wait of the tensor-memory kernel ran out
     # reconstruction alone, from the oracle's message (isolates the second kernel)
     ctx.core_set_round(t)
     gt3 = ctx.core_reconstruct(torch.from_numpy(pbaro.astype(np.float32)).cuda())
@@ -76,13 +77,18 @@ def test_ragged_sizes(core_mod, d, m, n):
     (11, 64, 9_001, "f32", "scaled_normal"),
     (9, 200, 70_000, "f32", "normal"),
     (25, 72, 3_000, "f32", "normal"),            # two tensor-core passes: 16 machines, then 9
+    (16, 256, 20_003, "bf16", "student_t3"),     # 9..16 machines and m >= 96: the tensor-memory (tcgen05) projection
+    (12, 1024, 5_003, "f32", "normal"),          # more CTA rows than coordinate tiles per column
+    (16, 384, 40_001, "f32", "scaled_normal"),
+    (10, 200, 300, "bf16", "normal"),            # a single ragged tile; last CTA row 72 of 128 vectors
+    (41, 128, 2_049, "f32", "normal"),           # three passes, the last one scalar
 ])
 def test_medium_sizes(core_mod, n, m, d, dtype, dist):
     G = core_inputs.gradients(n, d, seed=11, dist=dist, dtype=dtype, device="cuda")
     check_round(core_mod, G, m, seed=5, t=1)
 
 
-@pytest.mark.parametrize("n,d,m", [(3, 5003, 7), (10, 3001, 70)])     # scalar and tensor-core projection
+@pytest.mark.parametrize("n,d,m", [(3, 5003, 7), (10, 3001, 70), (13, 3001, 256)])   # scalar, warp-level and tcgen05 projection
 def test_unaligned_rows_and_leading_dimension(core_mod, n, d, m):
     for dtype in ("f32", "bf16"):
         # ld > d with an odd stride, and a base pointer that is not 16-byte aligned
@@ -92,13 +98,20 @@ def test_unaligned_rows_and_leading_dimension(core_mod, n, d, m):
         check_round(core_mod, G, m, seed=8, t=0)
 
 
-def test_bitwise_reproducible(core_mod):
-    G = core_inputs.gradients(8, 300_000, seed=4, device="cuda")
-    ctx = core_mod.Core(1, G.shape[1], 64)
+@pytest.mark.parametrize("n,m", [(8, 64), (16, 256)])                 # scalar and tcgen05 projection
+def test_bitwise_reproducible(core_mod, n, m):
+    G = core_inputs.gradients(n, 300_000, seed=4, device="cuda")
+    ctx = core_mod.Core(1, G.shape[1], m)
     a = ctx.core_round(G)
     ctx.core_set_round(0)
     b = ctx.core_round(G)
     assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+def test_device_status_word(core_mod):
+    import ctypes
+    assert core_mod.core_device_status() == 0
+    assert core_mod.lib().core_device_status(None) == -1        # CORE_EINVAL
 
 
 def test_round_index_and_seed_change_the_vectors(core_mod):
