@@ -252,8 +252,16 @@ static int round_with_epilogue(core_ctx *ctx, const void *G_dev, int dtype, int3
     if (int rc = ensure_workspace(ctx, pb + Pb)) return rc;
     float *partial = static_cast<float *>(ctx->ws);
     float *P = reinterpret_cast<float *>(static_cast<char *>(ctx->ws) + pb);
-    if (int rc = project_into(ctx, G_dev, dtype, n, ldg, ctx->d, 0, partial, P, false, ctx->stream)) return rc;
-    CORE_CUDA(ctx, launch_aggregate(P, n, ctx->m, pbar_dev, ctx->stream));
+    if (n <= kMaxGroup) {
+        // one group of machines: the per-machine messages are not kept, so they are never written
+        const ProjectPlan plan = make_project_plan(n, ctx->m, ctx->d, dtype, ctx->sm_count);
+        CORE_CUDA(ctx, launch_project(plan, ctx->keys, ctx->t, G_dev, dtype, n, ldg, ctx->d, ctx->m, 0, partial,
+                                      ctx->stream));
+        CORE_CUDA(ctx, launch_finish_aggregate(partial, plan.grid_x, n, ctx->m, pbar_dev, ctx->stream));
+    } else {
+        if (int rc = project_into(ctx, G_dev, dtype, n, ldg, ctx->d, 0, partial, P, false, ctx->stream)) return rc;
+        CORE_CUDA(ctx, launch_aggregate(P, n, ctx->m, pbar_dev, ctx->stream));
+    }
     CORE_CUDA(ctx, launch_reconstruct(ctx->keys, ctx->t, pbar_dev, ctx->m, 0, ctx->d, out, ctx->sm_count, ctx->stream,
                                       epilogue));
     ctx->t += 1;

@@ -58,6 +58,10 @@ cudaError_t launch_project(const ProjectPlan &plan, const RoundKeys &keys, uint3
 cudaError_t launch_finish_project(const float *partial, int chunks, int32_t n, int32_t m, float *P,
                                   bool accumulate, cudaStream_t stream);
 
+// pbar[j] = (1/n) sum_i (sum_c partial[c][i][j]): finish + aggregate for one group of machines, same order.
+cudaError_t launch_finish_aggregate(const float *partial, int chunks, int32_t n, int32_t m, float *pbar,
+                                    cudaStream_t stream);
+
 cudaError_t launch_aggregate(const float *P, int32_t n, int32_t m, float *pbar, cudaStream_t stream);
 
 // out[k - k_begin] = gtilde[k] for k in [k_begin, k_end); k_begin must be a multiple of 2048.

@@ -19,6 +19,9 @@ namespace core {
 namespace {
 
 __host__ __device__ constexpr int tile_q_for(int nb) { return nb <= 2 ? 1024 : 2048 / nb; }
+// Short vectors: with the tile above only a handful of CTAs would get work (d = 8192 is 8 tiles for
+// 8 machines), so small problems are cut into tiles of 32 blocks instead.
+constexpr int kSmallTileQ = 32;
 
 struct ProjectArgs {
     const void *G;
@@ -52,15 +55,14 @@ __device__ __forceinline__ float load_elem(const __nv_bfloat16 *p) {
     return __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short *>(p)) << 16);
 }
 
-template <int NB, int JT, int UQ, typename GT>
+template <int NB, int JT, int UQ, int TILE_Q, typename GT>
 __global__ void __launch_bounds__(kThreads, 2)
 project_kernel(const __grid_constant__ ProjectArgs a) {
-    constexpr int TILE_Q = tile_q_for(NB);
     constexpr int TILE = 4 * TILE_Q;
     constexpr bool BF16 = sizeof(GT) == 2;
     constexpr int PIECES = NB * TILE_Q / (BF16 ? 2 : 1);          // 16-byte pieces per tile
-    constexpr int PIECES_PER_THREAD = PIECES / kThreads;
-    static_assert(PIECES % kThreads == 0, "tile must split evenly over the CTA");
+    constexpr int PIECES_PER_THREAD = (PIECES + kThreads - 1) / kThreads;
+    constexpr bool EVEN = PIECES % kThreads == 0;                 // otherwise the last round is partial
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float4 *stage0 = reinterpret_cast<float4 *>(smem_raw);
@@ -98,6 +100,7 @@ project_kernel(const __grid_constant__ ProjectArgs a) {
 #pragma unroll
         for (int r = 0; r < PIECES_PER_THREAD; ++r) {
             const int piece = tid + r * kThreads;
+            if (!EVEN && piece >= PIECES) break;
             if constexpr (BF16) {
                 const int i = piece / (TILE_Q / 2);
                 const int c = piece % (TILE_Q / 2);
@@ -119,6 +122,7 @@ project_kernel(const __grid_constant__ ProjectArgs a) {
 #pragma unroll
                 for (int r = 0; r < PIECES_PER_THREAD; ++r) {
                     const int piece = tid + r * kThreads;
+                    if (!EVEN && piece >= PIECES) break;
                     const uint4 h = held[r];
                     // a bf16 is the upper half of an fp32
                     stage[2 * piece] = make_float4(__uint_as_float(h.x << 16), __uint_as_float(h.x & 0xFFFF0000u),
@@ -224,8 +228,8 @@ project_kernel(const __grid_constant__ ProjectArgs a) {
     }
 }
 
-template <int NB, int JT, int UQ>
-cudaError_t launch_typed(const ProjectPlan &plan, const ProjectArgs &args, int dtype, cudaStream_t stream) {
+template <int NB, int JT, int UQ, int TILE_Q>
+cudaError_t launch_tiled(const ProjectPlan &plan, const ProjectArgs &args, int dtype, cudaStream_t stream) {
     dim3 grid(plan.grid_x, plan.grid_y);
     auto go = [&](auto kernel) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem);
@@ -233,8 +237,14 @@ cudaError_t launch_typed(const ProjectPlan &plan, const ProjectArgs &args, int d
         kernel<<<grid, kThreads, plan.smem, stream>>>(args);
         return cudaGetLastError();
     };
-    if (dtype == 1) return go(project_kernel<NB, JT, UQ, __nv_bfloat16>);
-    return go(project_kernel<NB, JT, UQ, float>);
+    if (dtype == 1) return go(project_kernel<NB, JT, UQ, TILE_Q, __nv_bfloat16>);
+    return go(project_kernel<NB, JT, UQ, TILE_Q, float>);
+}
+
+template <int NB, int JT, int UQ>
+cudaError_t launch_typed(const ProjectPlan &plan, const ProjectArgs &args, int dtype, cudaStream_t stream) {
+    if (plan.tile_q == kSmallTileQ) return launch_tiled<NB, JT, UQ, kSmallTileQ>(plan, args, dtype, stream);
+    return launch_tiled<NB, JT, UQ, tile_q_for(NB)>(plan, args, dtype, stream);
 }
 
 __global__ void finish_project_kernel(const float *__restrict__ partial, int chunks, int n, int m,
@@ -252,6 +262,24 @@ __global__ void aggregate_kernel(const float *__restrict__ P, int n, int m, floa
     if (j >= m) return;
     float s = 0.f;
     for (int i = 0; i < n; ++i) s += P[(int64_t)i * m + j];
+    pbar[j] = s / (float)n;
+}
+
+// Both of the above in one launch for a single group of machines whose messages nobody asks for:
+// the same sums in the same order, so pbar is bitwise what the two kernels give.
+__global__ void finish_aggregate_kernel(const float *__restrict__ partial, int chunks, int n, int m,
+                                        float *__restrict__ pbar) {
+    __shared__ float message[kMaxGroup][32];       // P[i][j] of this block's 32 vectors
+    const int j = blockIdx.x * 32 + threadIdx.x, i = threadIdx.y;
+    const int64_t total = (int64_t)n * m;
+    float p = 0.f;
+    if (j < m && i < n)
+        for (int c = 0; c < chunks; ++c) p += partial[(int64_t)c * total + (int64_t)i * m + j];
+    message[i][threadIdx.x] = p;
+    __syncthreads();
+    if (i != 0 || j >= m) return;
+    float s = 0.f;
+    for (int r = 0; r < n; ++r) s += message[r][threadIdx.x];
     pbar[j] = s / (float)n;
 }
 
@@ -279,6 +307,13 @@ ProjectPlan make_project_plan(int32_t n_group, int32_t m, int64_t d, int dtype, 
     p.jt = (p.nb >= 8) ? 2 : 4;
     p.uq = (p.nb == 8) ? 2 : 1;
     p.tile_q = tile_q_for(p.nb);
+    {
+        // would the large tiles leave most SMs without a CTA?
+        const int tj_big = m >= kThreads * p.jt ? kThreads : 0;   // grid_y > 1 only then
+        const int64_t gy = tj_big ? (m + kThreads * p.jt - 1) / (kThreads * p.jt) : 1;
+        const int64_t tiles_big = (d + 4 * (int64_t)p.tile_q - 1) / (4 * (int64_t)p.tile_q);
+        if (tiles_big * gy < 2 * (int64_t)sm_count) p.tile_q = kSmallTileQ;
+    }
     int want = (m + p.jt - 1) / p.jt;                 // threads needed across vectors
     int tj = 1;
     while (tj < want && tj < kThreads) tj *= 2;
@@ -337,6 +372,12 @@ cudaError_t launch_finish_project(const float *partial, int chunks, int32_t n, i
     const int threads = 128;
     finish_project_kernel<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
         partial, chunks, n, m, P, accumulate ? 1 : 0);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_finish_aggregate(const float *partial, int chunks, int32_t n, int32_t m, float *pbar,
+                                    cudaStream_t stream) {
+    finish_aggregate_kernel<<<(m + 31) / 32, dim3(32, kMaxGroup), 0, stream>>>(partial, chunks, n, m, pbar);
     return cudaGetLastError();
 }
 

@@ -32,9 +32,10 @@ struct ReconstructArgs {
 constexpr int kRecJStep = 2;                      // vectors generated together per loop step
 
 // acc[u] += sum over JS consecutive table entries of pbar[j] * xi_j[block u], j ascending.
-template <int JS>
-__device__ __forceinline__ void rec_step(const uint4 *entries, const QPart (&qp)[kRecUQ], const RoundKeys &keys,
-                                         float4 (&acc)[kRecUQ]) {
+template <int JS, int UQ>
+__device__ __forceinline__ void rec_step(const uint4 *entries, const QPart (&qp)[UQ], const RoundKeys &keys,
+                                         float4 (&acc)[UQ]) {
+    constexpr int kRecUQ = UQ;
     uint4 w[JS * kRecUQ];
     float p[JS];
 #pragma unroll
@@ -58,6 +59,38 @@ __device__ __forceinline__ void rec_step(const uint4 *entries, const QPart (&qp)
             const float2 lo = __ffma2_rn(make_float2(p[s], p[s]), make_float2(zz.x, zz.y), make_float2(acc[u].x, acc[u].y));
             const float2 hi = __ffma2_rn(make_float2(p[s], p[s]), make_float2(zz.z, zz.w), make_float2(acc[u].z, acc[u].w));
             acc[u] = make_float4(lo.x, lo.y, hi.x, hi.y);
+        }
+    }
+}
+
+// The estimate r of block q goes out (or the update built from it, with an epilogue): one 16-byte
+// store where alignment allows, element by element on the ragged last block.
+__device__ __forceinline__ void emit_block(const ReconstructArgs &a, uint64_t q, uint64_t q_begin, float4 r) {
+    const int64_t off = (int64_t)((q - q_begin) << 2);        // offset into out
+    const int64_t k = (int64_t)(q << 2);
+    if (a.vec_ok && k + 4 <= a.k_end) {
+        float4 v = r;
+        if (a.epi.base) {
+            const float4 b = *reinterpret_cast<const float4 *>(a.epi.base + off);
+            v = make_float4(fmaf(-a.epi.step, r.x, b.x), fmaf(-a.epi.step, r.y, b.y),
+                            fmaf(-a.epi.step, r.z, b.z), fmaf(-a.epi.step, r.w, b.w));
+            if (a.epi.shift_dst) {
+                const float4 s = *reinterpret_cast<const float4 *>(a.epi.shift_src + off);
+                *reinterpret_cast<float4 *>(a.epi.shift_dst + off) = s;
+            }
+        }
+        *reinterpret_cast<float4 *>(a.out + off) = v;
+    } else {
+        const float vals[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+            if (k + l >= a.k_end) continue;
+            float v = vals[l];
+            if (a.epi.base) {
+                v = fmaf(-a.epi.step, v, a.epi.base[off + l]);
+                if (a.epi.shift_dst) a.epi.shift_dst[off + l] = a.epi.shift_src[off + l];
+            }
+            a.out[off + l] = v;
         }
     }
 }
@@ -105,42 +138,57 @@ reconstruct_kernel(const __grid_constant__ ReconstructArgs a) {
             }
             // kRecJStep vectors x kRecUQ blocks are generated together (one near-one test for all)
             int jj = 0;
-            for (; jj + kRecJStep <= jn; jj += kRecJStep) rec_step<kRecJStep>(table + jj, qp, a.keys, acc);
-            for (; jj < jn; ++jj) rec_step<1>(table + jj, qp, a.keys, acc);
+            for (; jj + kRecJStep <= jn; jj += kRecJStep) rec_step<kRecJStep, kRecUQ>(table + jj, qp, a.keys, acc);
+            for (; jj < jn; ++jj) rec_step<1, kRecUQ>(table + jj, qp, a.keys, acc);
         }
 
 #pragma unroll
         for (int u = 0; u < kRecUQ; ++u) {
             if (qv[u] >= q_end) continue;
-            const float4 r = make_float4(acc[u].x * inv_m, acc[u].y * inv_m, acc[u].z * inv_m, acc[u].w * inv_m);
-            const int64_t off = (int64_t)((qv[u] - q_begin) << 2);        // offset into out
-            const int64_t k = (int64_t)(qv[u] << 2);
-            if (a.vec_ok && k + 4 <= a.k_end) {
-                float4 v = r;
-                if (a.epi.base) {
-                    const float4 b = *reinterpret_cast<const float4 *>(a.epi.base + off);
-                    v = make_float4(fmaf(-a.epi.step, r.x, b.x), fmaf(-a.epi.step, r.y, b.y),
-                                    fmaf(-a.epi.step, r.z, b.z), fmaf(-a.epi.step, r.w, b.w));
-                    if (a.epi.shift_dst) {
-                        const float4 s = *reinterpret_cast<const float4 *>(a.epi.shift_src + off);
-                        *reinterpret_cast<float4 *>(a.epi.shift_dst + off) = s;
-                    }
-                }
-                *reinterpret_cast<float4 *>(a.out + off) = v;
-            } else {
-                const float vals[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-                for (int l = 0; l < 4; ++l) {
-                    if (k + l >= a.k_end) continue;
-                    float v = vals[l];
-                    if (a.epi.base) {
-                        v = fmaf(-a.epi.step, v, a.epi.base[off + l]);
-                        if (a.epi.shift_dst) a.epi.shift_dst[off + l] = a.epi.shift_src[off + l];
-                    }
-                    a.out[off + l] = v;
-                }
-            }
+            emit_block(a, qv[u], q_begin, make_float4(acc[u].x * inv_m, acc[u].y * inv_m, acc[u].z * inv_m, acc[u].w * inv_m));
         }
+    }
+}
+
+// Short vectors: the kernel above would give work to a handful of CTAs only (d = 8192 is four groups),
+// so here a CTA takes 32 blocks and its eight warps share out the vectors; the eight partial sums of a
+// block meet in shared memory and are added in ascending order of the vector ranges.
+constexpr int kSmallQ = 32;                        // blocks per CTA
+constexpr int kSmallSlices = kThreads / kSmallQ;   // ranges of vectors = warps
+
+__global__ void __launch_bounds__(kThreads)
+reconstruct_small_kernel(const __grid_constant__ ReconstructArgs a) {
+    __shared__ uint4 table[kJChunk];               // as above; m <= kJChunk here
+    __shared__ float4 part[kSmallSlices][kSmallQ];
+    const int tid = threadIdx.x, lane = tid & 31, slice = tid >> 5;
+    const uint64_t q_begin = (uint64_t)a.k_begin >> 2;
+    const uint64_t q_end = ((uint64_t)a.k_end + 3) >> 2;
+    const uint64_t q0 = q_begin + (uint64_t)blockIdx.x * kSmallQ;   // multiple of 32: one high counter word per CTA
+    const uint32_t q_hi = (uint32_t)(q0 >> 32);
+    for (int jj = tid; jj < a.m; jj += kThreads) {
+        const JPart jp = philox_jpart((uint32_t)jj, q_hi, a.keys);
+        table[jj] = make_uint4(jp.x0, jp.x2, jp.w3, __float_as_uint(a.pbar[jj]));
+    }
+    __syncthreads();
+    const uint64_t q = q0 + (uint64_t)lane;
+    QPart qp[1] = {philox_qpart((uint32_t)q, a.t, a.keys)};
+    float4 acc[1] = {make_float4(0.f, 0.f, 0.f, 0.f)};
+    const int per = ((a.m + kSmallSlices - 1) / kSmallSlices + 3) & ~3;   // vectors per warp, a multiple of 4
+    const int j_begin = min(slice * per, a.m), j_end = min(j_begin + per, a.m);
+    int jj = j_begin;
+    for (; jj + 4 <= j_end; jj += 4) rec_step<4, 1>(table + jj, qp, a.keys, acc);
+    for (; jj < j_end; ++jj) rec_step<1, 1>(table + jj, qp, a.keys, acc);
+    part[slice][lane] = acc[0];
+    __syncthreads();
+    if (slice == 0 && q < q_end) {
+        float4 s = part[0][lane];
+#pragma unroll
+        for (int r = 1; r < kSmallSlices; ++r) {
+            const float4 p = part[r][lane];
+            s = make_float4(s.x + p.x, s.y + p.y, s.z + p.z, s.w + p.w);
+        }
+        const float inv_m = 1.0f / (float)a.m;
+        emit_block(a, q, q_begin, make_float4(s.x * inv_m, s.y * inv_m, s.z * inv_m, s.w * inv_m));
     }
 }
 
@@ -216,6 +264,10 @@ cudaError_t launch_reconstruct(const RoundKeys &keys, uint32_t t, const float *p
     a.keys = keys;
     const int64_t nq = ((k_end + 3) >> 2) - (k_begin >> 2);
     const int64_t groups = (nq + kGroupQ - 1) / kGroupQ;
+    if (groups < sm_count && m <= kJChunk) {    // too few groups to go round: 32 blocks per CTA instead
+        reconstruct_small_kernel<<<(unsigned)((nq + kSmallQ - 1) / kSmallQ), kThreads, 0, stream>>>(a);
+        return cudaGetLastError();
+    }
     int64_t grid = (int64_t)sm_count * 3;     // three resident CTAs per SM (register-limited)
     if (grid > groups) grid = groups;
     reconstruct_kernel<<<(unsigned)grid, kThreads, 0, stream>>>(a);
