@@ -64,7 +64,9 @@ def test_ragged_sizes(core_mod, d, m, n):
 
 
 @pytest.mark.parametrize("n,m,d,dtype,dist", [
-    (2, 8, 200_003, "f32", "normal"),            # several tiles per CTA column, ragged tail
+    (2, 8, 200_003, "f32", "normal"),            # short-vector plans: 32-block tiles, vectors shared among warps
+    (2, 8, 1_300_003, "f32", "normal"),          # long-vector plans: several large tiles per CTA column, ragged tail
+    (8, 64, 400_003, "bf16", "scaled_normal"),
     (8, 64, 65_537, "f32", "scaled_normal"),
     (16, 40, 33_000, "bf16", "student_t3"),
     (17, 5, 20_001, "f32", "normal"),            # more than one machine group
