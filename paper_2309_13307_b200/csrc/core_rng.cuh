@@ -142,12 +142,12 @@ __device__ __forceinline__ uint4 philox_combine(const JPart &jp, const QPart &qp
 // (v is exact) the series of -log2(1 - v) replaces it.  That case is rare (one radius in
 // 1024), so it sits behind a branch tested once per call.
 //
-// Angle.  theta = 2 pi u = pi (h + y): adding a quarter turn to the word (an integer add
-// that wraps with the circle) puts the parity of h = round(2u) in bit 31 and the 22
-// fraction bits of y + 1/2 in bits 30..9.  Those bits, doubled plus one, inserted under
-// the exponent of 1.0, minus 1.5, are y in (-1/2, 1/2) exactly.  Then
-// (cos, sin) theta = (-1)^h (cos, sin)(pi y): odd/even minimax polynomials in y, and bit 31
-// is xored into the sign of S.
+// Angle.  theta = 2 pi u = pi (h + f) with h = bit 31 of the word (which half turn) and
+// f = (bits 30..9 + 1/2) / 2^22 in (0, 1).  Those 22 bits, doubled plus one, inserted under
+// the exponent of 1.0, minus 1.5, are y = f - 1/2 in (-1/2, 1/2) exactly, and
+//   cos theta = -(-1)^h sin(pi y),   sin theta = (-1)^h cos(pi y):
+// odd/even minimax polynomials in y (the minus sits in the odd one's coefficients), and bit
+// 31 is xored into the sign of S.  No integer arithmetic on the word beyond the bit insert.
 //
 // Worst absolute error over all 2^23 radius words and all 2^23 angle words: 1.2e-6.
 
@@ -187,25 +187,25 @@ __device__ __forceinline__ float4 bm_finish(uint4 w, float2 l) {
     asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(s.x) : "f"(fabsf(l.x)));
     asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(s.y) : "f"(fabsf(l.y)));
 
-    // angles
-    const uint32_t ra = w.y + 0x40000000u, rb = w.w + 0x40000000u;
-    const float2 y = __fadd2_rn(make_float2(__uint_as_float(((ra >> 8) & 0x007FFFFEu) | 0x3F800001u),
-                                            __uint_as_float(((rb >> 8) & 0x007FFFFEu) | 0x3F800001u)),
+    // angles: theta = pi (h + f), h = bit 31 of the word, f = (bits 30..9 + 1/2) / 2^22 in (0, 1).
+    // With y = f - 1/2:  cos theta = -(-1)^h sin(pi y),  sin theta = (-1)^h cos(pi y).
+    const float2 y = __fadd2_rn(make_float2(__uint_as_float(((w.y >> 8) & 0x007FFFFEu) | 0x3F800001u),
+                                            __uint_as_float(((w.w >> 8) & 0x007FFFFEu) | 0x3F800001u)),
                                 bm_splat(-1.5f));
-    s.x = __uint_as_float(__float_as_uint(s.x) ^ (ra & 0x80000000u));
-    s.y = __uint_as_float(__float_as_uint(s.y) ^ (rb & 0x80000000u));
+    s.x = __uint_as_float(__float_as_uint(s.x) ^ (w.y & 0x80000000u));
+    s.y = __uint_as_float(__float_as_uint(s.y) ^ (w.w & 0x80000000u));
     const float2 y2 = __fmul2_rn(y, y);
-    // sqrt(2 ln 2) sin(pi y) / y and sqrt(2 ln 2) cos(pi y)
-    float2 sp = __ffma2_rn(bm_splat(0.09091975539922714f), y2, bm_splat(-0.7041443586349487f));
-    sp = __ffma2_rn(sp, y2, bm_splat(3.0024325847625732f));
-    sp = __ffma2_rn(sp, y2, bm_splat(-6.08450984954834f));
-    sp = __ffma2_rn(sp, y2, bm_splat(3.6989426612854004f));
+    // -sqrt(2 ln 2) sin(pi y) / y and sqrt(2 ln 2) cos(pi y)
+    float2 sp = __ffma2_rn(bm_splat(-0.09091975539922714f), y2, bm_splat(0.7041443586349487f));
+    sp = __ffma2_rn(sp, y2, bm_splat(-3.0024325847625732f));
+    sp = __ffma2_rn(sp, y2, bm_splat(6.08450984954834f));
+    sp = __ffma2_rn(sp, y2, bm_splat(-3.6989426612854004f));
     float2 cp = __ffma2_rn(bm_splat(0.2591251730918884f), y2, bm_splat(-1.568420648574829f));
     cp = __ffma2_rn(cp, y2, bm_splat(4.778461456298828f));
     cp = __ffma2_rn(cp, y2, bm_splat(-5.810277938842773f));
     const float2 cs = __ffma2_rn(cp, y2, bm_splat(1.1774100065231323f));
-    const float2 zc = __fmul2_rn(s, cs);
-    const float2 zs = __fmul2_rn(__fmul2_rn(s, y), sp);
+    const float2 zs = __fmul2_rn(s, cs);                       // r sin theta
+    const float2 zc = __fmul2_rn(__fmul2_rn(s, y), sp);        // r cos theta
     return make_float4(zc.x, zs.x, zc.y, zs.y);
 }
 
