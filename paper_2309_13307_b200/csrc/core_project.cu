@@ -22,6 +22,9 @@ __host__ __device__ constexpr int tile_q_for(int nb) { return nb <= 2 ? 1024 : 2
 // Short vectors: with the tile above only a handful of CTAs would get work (d = 8192 is 8 tiles for
 // 8 machines), so small problems are cut into tiles of 32 blocks instead.
 constexpr int kSmallTileQ = 32;
+// In between, and for few vectors (a tile of 32 blocks keeps at least 8 threads across the vectors, which
+// idle when there are fewer than 8 x JT of them): tiles of 128 blocks.
+constexpr int kMediumTileQ = 128;
 
 struct ProjectArgs {
     const void *G;
@@ -244,6 +247,8 @@ cudaError_t launch_tiled(const ProjectPlan &plan, const ProjectArgs &args, int d
 template <int NB, int JT, int UQ>
 cudaError_t launch_typed(const ProjectPlan &plan, const ProjectArgs &args, int dtype, cudaStream_t stream) {
     if (plan.tile_q == kSmallTileQ) return launch_tiled<NB, JT, UQ, kSmallTileQ>(plan, args, dtype, stream);
+    if (plan.tile_q == kMediumTileQ && kMediumTileQ != tile_q_for(NB))
+        return launch_tiled<NB, JT, UQ, kMediumTileQ>(plan, args, dtype, stream);
     return launch_tiled<NB, JT, UQ, tile_q_for(NB)>(plan, args, dtype, stream);
 }
 
@@ -308,11 +313,18 @@ ProjectPlan make_project_plan(int32_t n_group, int32_t m, int64_t d, int dtype, 
     p.uq = (p.nb == 8) ? 2 : 1;
     p.tile_q = tile_q_for(p.nb);
     {
-        // would the large tiles leave most SMs without a CTA?
+        // would the large tiles leave SMs without a CTA, or give the CTAs too few tiles to share out evenly?
         const int tj_big = m >= kThreads * p.jt ? kThreads : 0;   // grid_y > 1 only then
         const int64_t gy = tj_big ? (m + kThreads * p.jt - 1) / (kThreads * p.jt) : 1;
         const int64_t tiles_big = (d + 4 * (int64_t)p.tile_q - 1) / (4 * (int64_t)p.tile_q);
-        if (tiles_big * gy < 2 * (int64_t)sm_count) p.tile_q = kSmallTileQ;
+        if (tiles_big * gy < 8 * (int64_t)sm_count) {
+            int tj_want = 1;
+            while (tj_want < (m + p.jt - 1) / p.jt && tj_want < kThreads) tj_want *= 2;
+            const bool small_fits = kThreads * p.uq / kSmallTileQ <= tj_want;      // no idle threads across vectors
+            const int64_t tiles_medium = (d + 4 * (int64_t)kMediumTileQ - 1) / (4 * (int64_t)kMediumTileQ);
+            const bool medium_fills = tiles_medium * gy >= sm_count / 2;
+            p.tile_q = (small_fits || !medium_fills || kMediumTileQ > p.tile_q) ? kSmallTileQ : kMediumTileQ;
+        }
     }
     int want = (m + p.jt - 1) / p.jt;                 // threads needed across vectors
     int tj = 1;

@@ -151,40 +151,40 @@ reconstruct_kernel(const __grid_constant__ ReconstructArgs a) {
 }
 
 // Short vectors: the kernel above would give work to a handful of CTAs only (d = 8192 is four groups),
-// so here a CTA takes 32 blocks and its eight warps share out the vectors; the eight partial sums of a
-// block meet in shared memory and are added in ascending order of the vector ranges.
-constexpr int kSmallQ = 32;                        // blocks per CTA
-constexpr int kSmallSlices = kThreads / kSmallQ;   // ranges of vectors = warps
-
+// so here the SLICES warp groups of a CTA share out the vectors of 256 / SLICES blocks; the partial sums
+// of a block meet in shared memory and are added in ascending order of the vector ranges.  Few vectors
+// get few slices (a slice wants at least four vectors to generate together).
+template <int SLICES>
 __global__ void __launch_bounds__(kThreads)
 reconstruct_small_kernel(const __grid_constant__ ReconstructArgs a) {
+    constexpr int QB = kThreads / SLICES;          // blocks per CTA
     __shared__ uint4 table[kJChunk];               // as above; m <= kJChunk here
-    __shared__ float4 part[kSmallSlices][kSmallQ];
-    const int tid = threadIdx.x, lane = tid & 31, slice = tid >> 5;
+    __shared__ float4 part[SLICES][QB];
+    const int tid = threadIdx.x, ql = tid % QB, slice = tid / QB;
     const uint64_t q_begin = (uint64_t)a.k_begin >> 2;
     const uint64_t q_end = ((uint64_t)a.k_end + 3) >> 2;
-    const uint64_t q0 = q_begin + (uint64_t)blockIdx.x * kSmallQ;   // multiple of 32: one high counter word per CTA
+    const uint64_t q0 = q_begin + (uint64_t)blockIdx.x * QB;     // multiple of 32: one high counter word per CTA
     const uint32_t q_hi = (uint32_t)(q0 >> 32);
     for (int jj = tid; jj < a.m; jj += kThreads) {
         const JPart jp = philox_jpart((uint32_t)jj, q_hi, a.keys);
         table[jj] = make_uint4(jp.x0, jp.x2, jp.w3, __float_as_uint(a.pbar[jj]));
     }
     __syncthreads();
-    const uint64_t q = q0 + (uint64_t)lane;
+    const uint64_t q = q0 + (uint64_t)ql;
     QPart qp[1] = {philox_qpart((uint32_t)q, a.t, a.keys)};
     float4 acc[1] = {make_float4(0.f, 0.f, 0.f, 0.f)};
-    const int per = ((a.m + kSmallSlices - 1) / kSmallSlices + 3) & ~3;   // vectors per warp, a multiple of 4
+    const int per = ((a.m + SLICES - 1) / SLICES + 3) & ~3;      // vectors per slice, a multiple of 4
     const int j_begin = min(slice * per, a.m), j_end = min(j_begin + per, a.m);
     int jj = j_begin;
     for (; jj + 4 <= j_end; jj += 4) rec_step<4, 1>(table + jj, qp, a.keys, acc);
     for (; jj < j_end; ++jj) rec_step<1, 1>(table + jj, qp, a.keys, acc);
-    part[slice][lane] = acc[0];
+    part[slice][ql] = acc[0];
     __syncthreads();
     if (slice == 0 && q < q_end) {
-        float4 s = part[0][lane];
+        float4 s = part[0][ql];
 #pragma unroll
-        for (int r = 1; r < kSmallSlices; ++r) {
-            const float4 p = part[r][lane];
+        for (int r = 1; r < SLICES; ++r) {
+            const float4 p = part[r][ql];
             s = make_float4(s.x + p.x, s.y + p.y, s.z + p.z, s.w + p.w);
         }
         const float inv_m = 1.0f / (float)a.m;
@@ -264,8 +264,18 @@ cudaError_t launch_reconstruct(const RoundKeys &keys, uint32_t t, const float *p
     a.keys = keys;
     const int64_t nq = ((k_end + 3) >> 2) - (k_begin >> 2);
     const int64_t groups = (nq + kGroupQ - 1) / kGroupQ;
-    if (groups < sm_count && m <= kJChunk) {    // too few groups to go round: 32 blocks per CTA instead
-        reconstruct_small_kernel<<<(unsigned)((nq + kSmallQ - 1) / kSmallQ), kThreads, 0, stream>>>(a);
+    if (groups < 8 * (int64_t)sm_count && m <= kJChunk) {    // too few groups to go round evenly: smaller units
+        // more slices = fewer blocks per CTA = more CTAs: as many as it takes to go round, while a slice
+        // keeps at least four vectors
+        int slices = 1;
+        while (slices < 8 && m >= 8 * slices && nq / (kThreads / slices) < 4 * (int64_t)sm_count) slices *= 2;
+        const unsigned grid = (unsigned)((nq + kThreads / slices - 1) / (kThreads / slices));
+        switch (slices) {
+            case 8: reconstruct_small_kernel<8><<<grid, kThreads, 0, stream>>>(a); break;
+            case 4: reconstruct_small_kernel<4><<<grid, kThreads, 0, stream>>>(a); break;
+            case 2: reconstruct_small_kernel<2><<<grid, kThreads, 0, stream>>>(a); break;
+            default: reconstruct_small_kernel<1><<<grid, kThreads, 0, stream>>>(a); break;
+        }
         return cudaGetLastError();
     }
     int64_t grid = (int64_t)sm_count * 3;     // three resident CTAs per SM (register-limited)
