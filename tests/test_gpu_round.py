@@ -206,6 +206,26 @@ def test_gpt2small_sized_bf16(core_mod):
     sampled_full_size(core_mod, "gpt2small", 1024, js=(511,), machines=(0, 15))
 
 
+@pytest.mark.parametrize("name,m", [("resnet50", 256), ("gpt2small", 1024)])
+def test_full_size_round_keeps_the_inner_product(core_mod, name, m):
+    """A property that holds at any size and involves every coordinate and every vector:
+    <gbar, gtilde> = (1/m) sum_j pbar_j <gbar, xi_j> = (1/m) sum_j pbar_j^2, with gbar the mean
+    gradient.  Projection and reconstruction must have regenerated the same vectors for it to hold."""
+    w = core_inputs.WORKLOADS[name]
+    G = core_inputs.workload_gradients(name, seed=0, device="cuda")
+    ctx = core_mod.Core(1, w.d, m)
+    pbar, gt = ctx.core_round(G)
+    assert core_mod.core_device_status() == 0
+    lhs = 0.0
+    step = 1 << 22
+    for k0 in range(0, w.d, step):                      # fp64 in chunks: the operands are large
+        gbar = G[:, k0:k0 + step].to(torch.float64).mean(dim=0)
+        lhs += float((gbar * gt[k0:k0 + step].to(torch.float64)).sum())
+    rhs = float((pbar.to(torch.float64) ** 2).sum()) / m
+    # fp32 accumulation leaves about 1e-7 of ||gtilde|| ~ ||gbar|| sqrt(d / m) in gtilde
+    assert abs(lhs - rhs) <= 5e-3 * rhs, (lhs, rhs)
+
+
 @pytest.mark.parametrize("m", [8, 4096])
 def test_sweep_sized(core_mod, m):
     sampled_full_size(core_mod, "sweep", m, js=(m - 1,), machines=(1,))
