@@ -155,6 +155,11 @@ project_kernel(const __grid_constant__ ProjectArgs a) {
     cp_async_wait_all();
     __syncthreads();
 
+    // the vector-dependent half of Philox changes only with the high word of the block index
+    JPart jp[JT];
+    uint32_t jp_q_hi = 0;
+    bool have_jp = false;
+
     for (int64_t tile = tile_begin; tile < tile_end; ++tile) {
         float4 *cur = ((tile - tile_begin) & 1) ? stage1 : stage0;
         float4 *nxt = ((tile - tile_begin) & 1) ? stage0 : stage1;
@@ -164,9 +169,12 @@ project_kernel(const __grid_constant__ ProjectArgs a) {
         const uint64_t q0 = a.q_base + (uint64_t)tile * TILE_Q;   // multiple of TILE_Q: no carry inside
         const uint32_t q0_lo = (uint32_t)q0;
         const uint32_t q_hi = (uint32_t)(q0 >> 32);
-        JPart jp[JT];
+        if (!have_jp || q_hi != jp_q_hi) {
 #pragma unroll
-        for (int v = 0; v < JT; ++v) jp[v] = philox_jpart((uint32_t)(jbase + jl + v * tj), q_hi, a.keys);
+            for (int v = 0; v < JT; ++v) jp[v] = philox_jpart((uint32_t)(jbase + jl + v * tj), q_hi, a.keys);
+            jp_q_hi = q_hi;
+            have_jp = true;
+        }
 
         float acc[NB][JT];
 #pragma unroll
