@@ -431,7 +431,7 @@ def run_leastsq(args):
         "metric": "least-squares CORE-GD step", "value": ms, "unit": "ms/step", "higher_is_better": False,
         "n_gpus": 1, "steps": steps, "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"leastsq: n={n}, A_i {rows}x{d} fp32 (|A| = {a_bytes} bytes, larger than L2), m={m}"},
-        "loss": float(ctx.core_ls_loss(ls, x).item()), "gpu_launches": 5 * steps,   # gradients (2), project, finish+aggregate, reconstruct+update
+        "loss": float(ctx.core_ls_loss(ls, x).item()), "gpu_launches": 4 * steps,   # gradient partials, project (sums them while staging), finish+aggregate, reconstruct+update
         "gradients_ms": grad_ms, "round_and_update_ms": ms - grad_ms,
         "roofline": {"bound": "hbm", "kernel": "ls_fused_kernel + ls_reduce_kernel", "achieved": achieved,
                      "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak, "traffic": None,

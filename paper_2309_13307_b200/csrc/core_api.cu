@@ -434,6 +434,30 @@ static int ls_gradients_into(core_ctx *ctx, core_ls *ls, const float *x_dev, flo
     return CORE_OK;
 }
 
+// Gradients at x_eval, then the round with the given epilogue.  Where the single-pass gradient kernel
+// and the scalar projection both apply, the projection sums the per-row-range partial gradients while
+// it stages its tiles, so the machine gradients G are never written or read back.
+static int ls_round(core_ctx *ctx, core_ls *ls, const float *x_eval, float *out, const ReconstructEpilogue *epilogue) {
+    if (ls->n <= kMaxGroup && ls_fused_usable(ls->fused_plan, ls->A, x_eval, ls->part)) {
+        const ProjectPlan plan = make_project_plan(ls->n, ctx->m, ctx->d, CORE_F32, ctx->sm_count);
+        if (plan.mma == 0) {
+            if (int rc = ensure_workspace(ctx, partial_bytes(ctx, ls->n, ctx->d, CORE_F32))) return rc;
+            float *partial = static_cast<float *>(ctx->ws);
+            CORE_CUDA(ctx, launch_ls_fused(ls->fused_plan, ls->A, ls->b, x_eval, ls->n, ls->rows, ls->d, ls->part,
+                                           ctx->stream));
+            CORE_CUDA(ctx, launch_project(plan, ctx->keys, ctx->t, ls->part, CORE_F32, ls->n, ls->d, ctx->d, ctx->m, 0,
+                                          partial, ctx->stream, ls->fused_plan.splits, 1.0f / (float)ls->rows));
+            CORE_CUDA(ctx, launch_finish_aggregate(partial, plan.grid_x, ls->n, ctx->m, ctx->pbar, ctx->stream));
+            CORE_CUDA(ctx, launch_reconstruct(ctx->keys, ctx->t, ctx->pbar, ctx->m, 0, ctx->d, out, ctx->sm_count,
+                                              ctx->stream, epilogue));
+            ctx->t += 1;
+            return CORE_OK;
+        }
+    }
+    if (int rc = ls_gradients_into(ctx, ls, x_eval, ls->G)) return rc;
+    return round_with_epilogue(ctx, ls->G, CORE_F32, ls->n, ls->d, ctx->pbar, out, epilogue);
+}
+
 int core_ls_gradients(core_ctx *ctx, core_ls *ls, const float *x_dev, float *G_out_dev) {
     if (int rc = check_ctx(ctx)) return rc;
     if (!ls || !x_dev || !G_out_dev || ls->d != ctx->d || ls->device != ctx->device) return CORE_EINVAL;
@@ -443,10 +467,9 @@ int core_ls_gradients(core_ctx *ctx, core_ls *ls, const float *x_dev, float *G_o
 int core_gd_step(core_ctx *ctx, core_ls *ls, float h, float *x_dev) {
     if (int rc = check_ctx(ctx)) return rc;
     if (!ls || !x_dev || ls->d != ctx->d || ls->device != ctx->device) return CORE_EINVAL;
-    if (int rc = ls_gradients_into(ctx, ls, x_dev, ls->G)) return rc;
     // x <- x - h * gtilde inside the reconstruction: the estimate is never stored
     const ReconstructEpilogue update{x_dev, h, nullptr, nullptr};
-    return round_with_epilogue(ctx, ls->G, CORE_F32, ls->n, ls->d, ctx->pbar, x_dev, &update);
+    return ls_round(ctx, ls, x_dev, x_dev, &update);
 }
 
 int core_agd_step(core_ctx *ctx, core_ls *ls, float h, float beta, float *x_dev, float *x_prev_dev) {
@@ -454,19 +477,17 @@ int core_agd_step(core_ctx *ctx, core_ls *ls, float h, float beta, float *x_dev,
     if (!ls || !x_dev || !x_prev_dev || x_dev == x_prev_dev || ls->d != ctx->d || ls->device != ctx->device)
         return CORE_EINVAL;
     CORE_CUDA(ctx, launch_lookahead(x_dev, x_prev_dev, 1.0f - beta, ls->d, ls->y, ctx->stream));
-    if (int rc = ls_gradients_into(ctx, ls, ls->y, ls->G)) return rc;
     // x_prev <- x and x <- y - h * gtilde(y), both inside the reconstruction
     const ReconstructEpilogue update{ls->y, h, x_dev, x_prev_dev};
-    return round_with_epilogue(ctx, ls->G, CORE_F32, ls->n, ls->d, ctx->pbar, x_dev, &update);
+    return ls_round(ctx, ls, ls->y, x_dev, &update);
 }
 
 int core_gd_step_guarded(core_ctx *ctx, core_ls *ls, float h, float *x_dev, double *f_dev, int32_t *accepted_dev) {
     if (int rc = check_ctx(ctx)) return rc;
     if (!ls || !x_dev || !f_dev || ls->d != ctx->d || ls->device != ctx->device) return CORE_EINVAL;
-    if (int rc = ls_gradients_into(ctx, ls, x_dev, ls->G)) return rc;
     // trial point y = x - h * gtilde, written by the reconstruction; x is left untouched
     const ReconstructEpilogue trial{x_dev, h, nullptr, nullptr};
-    if (int rc = round_with_epilogue(ctx, ls->G, CORE_F32, ls->n, ls->d, ctx->pbar, ls->y, &trial)) return rc;
+    if (int rc = ls_round(ctx, ls, x_dev, ls->y, &trial)) return rc;
     CORE_CUDA(ctx, launch_ls_residual(ls->A, ls->b, ls->y, ls->n, ls->rows, ls->d, ls->res, ctx->stream));
     CORE_CUDA(ctx, launch_ls_loss(ls->res, ls->n, ls->rows, ls->f_trial, ctx->stream));
     // decided on the device: no host synchronisation inside the step

@@ -50,9 +50,12 @@ cudaError_t project_tc_take_status(int *status);
 // One projection pass over coordinates [0, d) of rows G + i*ldg, i < n <= 16.
 // q_base is the global index of the block holding coordinate 0 of G (non-zero when G
 // is a slab of a longer vector).  Writes partial[(c * n + i) * m + j], c < plan.grid_x.
+// With splits > 0 (fp32, scalar kernel only: plan.mma == 0) row i is not stored anywhere: it is
+// scale * (G[(i*splits + 0)*ldg + k] + ... + G[(i*splits + splits-1)*ldg + k]), summed in that order
+// while the tile is staged (the per-row-range partial gradients of the least-squares kernels).
 cudaError_t launch_project(const ProjectPlan &plan, const RoundKeys &keys, uint32_t t, const void *G,
                            int dtype, int32_t n, int64_t ldg, int64_t d, int32_t m, uint64_t q_base,
-                           float *partial, cudaStream_t stream);
+                           float *partial, cudaStream_t stream, int splits = 0, float scale = 1.0f);
 
 // P[i*m+j] = (accumulate ? P[i*m+j] : 0) + sum_c partial[c][i][j], c ascending.
 cudaError_t launch_finish_project(const float *partial, int chunks, int32_t n, int32_t m, float *P,

@@ -38,6 +38,8 @@ struct ProjectArgs {
     int tj;          // threads across vectors
     int tj_log2;
     int aligned;     // rows may be copied in 16-byte pieces
+    int splits;      // > 0: row i is the sum of `splits` arrays ldg apart, times `scale` (see launch_project)
+    float scale;
     uint32_t t;
     RoundKeys keys;
 };
@@ -136,9 +138,32 @@ project_kernel(const __grid_constant__ ProjectArgs a) {
             }
             return;
         }
-        // ragged or unaligned tile: element by element, zero beyond d and beyond n
         float *flat = reinterpret_cast<float *>(stage);
         const int64_t k0 = tile * TILE;
+        if constexpr (!BF16) {
+            if (a.splits > 0) {
+                // summed rows (d and ldg are multiples of 4 here): one block of four coordinates per thread
+                // step, the `splits` 16-byte loads of a block independent of one another
+                for (int e = tid; e < NB * TILE_Q; e += kThreads) {
+                    const int i = e / TILE_Q;
+                    const int64_t k = k0 + 4 * (e % TILE_Q);
+                    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (i < a.n && k < a.d) {
+                        const float4 *src = reinterpret_cast<const float4 *>(G + (int64_t)i * a.splits * a.ldg + k);
+                        const int64_t stride4 = a.ldg >> 2;
+#pragma unroll 6
+                        for (int c = 0; c < a.splits; ++c) {
+                            const float4 v = __ldg(src + (int64_t)c * stride4);
+                            sum = make_float4(sum.x + v.x, sum.y + v.y, sum.z + v.z, sum.w + v.w);
+                        }
+                        sum = make_float4(sum.x * a.scale, sum.y * a.scale, sum.z * a.scale, sum.w * a.scale);
+                    }
+                    stage[e] = sum;
+                }
+                return;
+            }
+        }
+        // ragged or unaligned tile: element by element, zero beyond d and beyond n
         for (int e = tid; e < NB * TILE; e += kThreads) {
             const int i = e / TILE;
             const int64_t k = k0 + (e % TILE);
@@ -359,7 +384,10 @@ ProjectPlan make_project_plan(int32_t n_group, int32_t m, int64_t d, int dtype, 
 
 cudaError_t launch_project(const ProjectPlan &plan, const RoundKeys &keys, uint32_t t, const void *G,
                            int dtype, int32_t n, int64_t ldg, int64_t d, int32_t m, uint64_t q_base,
-                           float *partial, cudaStream_t stream) {
+                           float *partial, cudaStream_t stream, int splits, float scale) {
+    if (splits > 0 && (plan.mma != 0 || dtype != 0 || d % 4 != 0 || ldg % 4 != 0 ||
+                       reinterpret_cast<uintptr_t>(G) % 16 != 0))
+        return cudaErrorInvalidValue;
     if (plan.mma == 2) return launch_project_tc(plan, keys, t, G, dtype, n, ldg, d, m, q_base, partial, stream);
     if (plan.mma == 1) return launch_project_mma(plan, keys, t, G, dtype, n, ldg, d, m, q_base, partial, stream);
     ProjectArgs a{};
@@ -375,6 +403,9 @@ cudaError_t launch_project(const ProjectPlan &plan, const RoundKeys &keys, uint3
     a.tj_log2 = ilog2(plan.tj);
     const size_t es = dtype == 1 ? 2 : 4;
     a.aligned = ((reinterpret_cast<uintptr_t>(G) % 16) == 0 && ((size_t)ldg * es) % 16 == 0) ? 1 : 0;
+    a.splits = splits;
+    a.scale = scale;
+    if (splits > 0) a.aligned = 0;      // summed rows are formed element by element while the tile is staged
     a.t = t;
     a.keys = keys;
     switch (plan.nb) {
