@@ -21,11 +21,16 @@ import sys
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
+# The files project_kernel and reconstruct_kernel (the two kernels the DRAM capture covers) are compiled from.
+ROUND_KERNEL_SOURCES = ("core_internal.h", "core_project.cu", "core_reconstruct.cu", "core_rng.cuh")
+
+
 def csrc_digest() -> str:
+    """Digest of the sources of the two captured kernels: the stored counters describe exactly this code."""
     h = hashlib.sha256()
-    for path in sorted(glob.glob(os.path.join(ROOT, "paper_2309_13307_b200", "csrc", "*"))):
-        h.update(os.path.basename(path).encode())
-        h.update(open(path, "rb").read())
+    for name in ROUND_KERNEL_SOURCES:
+        h.update(name.encode())
+        h.update(open(os.path.join(ROOT, "paper_2309_13307_b200", "csrc", name), "rb").read())
     return h.hexdigest()
 
 
