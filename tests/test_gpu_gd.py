@@ -70,3 +70,26 @@ def test_least_squares_workload_200_iterations(core_mod):
     ls_in = core_inputs.least_squares(n=8, rows=2048, d=8192, seed=0, device="cuda")
     gpu_loss, orc_loss = run_both(core_mod, ls_in, 64, 200)
     assert gpu_loss[-1] < 0.5 * gpu_loss[0]
+
+
+@pytest.mark.parametrize("n,rows,d,m", [(8, 256, 4096, 64), (3, 50, 1001, 8)])
+def test_step_equals_its_parts(core_mod, n, rows, d, m):
+    """core_gd_step never stores the machine gradients (where the single-pass gradient kernel applies the
+    projection adds their partial sums while it stages its tiles).  Building the same step from the entry
+    points that do store them - gradients, round, update - must give the same iterate: the sums are the same
+    and taken in the same order, so only the final multiply-add may round differently."""
+    ls_in = core_inputs.least_squares(n=n, rows=rows, d=d, seed=3, device="cuda")
+    h = 0.37
+    x0 = core_inputs.gradients(1, d, seed=5, device="cuda")[0].contiguous()
+    ls = core_mod.LeastSquares(ls_in.A, ls_in.b)
+    whole, parts = core_mod.Core(9, d, m), core_mod.Core(9, d, m)
+    whole.core_set_round(4)
+    parts.core_set_round(4)
+    x = x0.clone()
+    whole.core_gd_step(ls, h, x)
+    G = parts.core_ls_gradients(ls, x0)
+    _, gt = parts.core_round(G)
+    want = x0.double() - h * gt.double()
+    assert whole.core_get_round() == parts.core_get_round() == 5
+    err = (x.double() - want).abs().max().item()
+    assert err <= 2e-7 * max(1.0, want.abs().max().item()), err
