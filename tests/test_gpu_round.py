@@ -116,6 +116,42 @@ def test_device_status_word(core_mod):
     assert core_mod.lib().core_device_status(None) == -1        # CORE_EINVAL
 
 
+@pytest.mark.parametrize("n,m,dtype", [
+    (2, 8, "f32"), (4, 40, "bf16"), (8, 64, "f32"),       # scalar projection
+    (10, 70, "f32"), (12, 72, "bf16"),                    # warp-level tensor-core projection
+    (16, 256, "bf16"), (9, 128, "f32"),                   # tcgen05 projection
+])
+def test_unit_vectors_read_the_generator_back(core_mod, n, m, dtype):
+    """Machine i holds the unit vector e_k(i): its message is p_ij = xi_j[k(i)], and every other term of
+    the sum is an exact zero, so the scalar projection must return the generator's own fp32 values bit for
+    bit.  On the tensor-core paths the tail of a split value is itself cut to tf32, which leaves 2^-21 of
+    the value.  Likewise pbar = e_j reconstructs xi_j / m, bit for bit."""
+    d, seed, t = 70_001, 6, 3
+    ks = [(i * 7919 + 5) % d for i in range(n)]
+    ks[0], ks[-1] = 0, d - 1                               # first block, ragged last block
+    G = torch.zeros((n, d), dtype=torch.float32, device="cuda")
+    for i, k in enumerate(ks):
+        G[i, k] = 1.0
+    if dtype == "bf16":
+        G = G.to(torch.bfloat16)
+    ctx = core_mod.Core(seed, d, m)
+    ctx.core_set_round(t)
+    P = ctx.core_project(G)
+    assert core_mod.core_device_status() == 0
+    scalar = n <= 8
+    for j in sorted({0, 1, m // 2, m - 1}):
+        z = ctx.core_debug_gaussians(j, 0, (d + 3) // 4).reshape(-1)      # xi_j[0 .. 4 ceil(d/4))
+        for i, k in enumerate(ks):
+            got, want = P[i, j].item(), z[k].item()
+            assert got == want if scalar else abs(got - want) <= 2.0 ** -20 * abs(want), (i, j, k, got, want)
+    for j in sorted({0, m - 1}):
+        pbar = torch.zeros(m, dtype=torch.float32, device="cuda")
+        pbar[j] = 1.0
+        gt = ctx.core_reconstruct(pbar)
+        z = ctx.core_debug_gaussians(j, 0, (d + 3) // 4).reshape(-1)[:d]
+        assert torch.equal(gt, z * torch.tensor(1.0 / m, dtype=torch.float32, device="cuda")), j
+
+
 def test_round_index_and_seed_change_the_vectors(core_mod):
     G = core_inputs.gradients(2, 4096, seed=4, device="cuda")
     base = core_mod.Core(1, 4096, 8).core_project(G)
