@@ -184,9 +184,10 @@ def test_host_round_matches_oracle_and_device_round(core_mod):
     assert rel_l2(gt_h.numpy(), gt_d.cpu().numpy()) <= REC_TOL
 
 
-def test_host_round_many_slabs(core_mod):
+@pytest.mark.parametrize("m", [8, 128])      # scalar and tcgen05 projection (slabs start at non-zero blocks)
+def test_host_round_many_slabs(core_mod, m):
     # bf16, 16 machines: slabs of 2^21 coordinates, so d = 5e6 + 3 takes three slabs
-    n, d, m = 16, 5_000_003, 8
+    n, d = 16, 5_000_003
     G = core_inputs.gradients(n, d, seed=3, dtype="bf16", dist="student_t3", device="cuda")
     Gh = G.cpu()
     ctx = core_mod.Core(4, d, m)
