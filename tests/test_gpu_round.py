@@ -263,6 +263,6 @@ def test_full_size_round_keeps_the_inner_product(core_mod, name, m):
     assert abs(lhs - rhs) <= 5e-3 * rhs, (lhs, rhs)
 
 
-@pytest.mark.parametrize("m", [8, 4096])
+@pytest.mark.parametrize("m", [8, 64, 512, 4096])      # every launch plan of the sweep (tj = 2, 16, 128, 256)
 def test_sweep_sized(core_mod, m):
     sampled_full_size(core_mod, "sweep", m, js=(m - 1,), machines=(1,))

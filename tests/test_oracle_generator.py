@@ -185,3 +185,42 @@ def test_vectors_and_rounds_are_fresh():
                   oracle.xi_range(6, 0, 0, 0, 1 << 16)):
         assert abs(np.corrcoef(base, other)[0, 1]) < 5 / math.sqrt(base.size)
     assert np.array_equal(base, oracle.xi_range(5, 0, 0, 0, 1 << 16))
+
+
+# ---- the two loop helpers the GPU generator tests take their expected values from ------------
+
+def test_xi_words_range_is_xi_words_block_by_block():
+    # a window that starts away from zero and crosses a multiple of 2^32 (the high counter word
+    # changes inside it): row r must be the words of block q0 + r, not of block r or q0 + r +- 1
+    for seed, t, j, q0, nq in [(0xDEADBEEFCAFEF00D, 7, 4095, (1 << 32) - 37, 80), (5, 2, 1, 12345, 50),
+                               (3, 0, 5, 0, 16), (2**64 - 1, 2**32 - 1, 2**32 - 1, (1 << 40) + 3, 9)]:
+        W = oracle.xi_words_range(seed, t, j, q0, q0 + nq)
+        assert W.shape == (nq, 4) and W.dtype == np.uint32
+        for r in range(nq):
+            q = q0 + r
+            assert [int(x) for x in W[r]] == bigint_philox([q & MASK, q >> 32, j, t], [seed & MASK, seed >> 32])
+            assert np.array_equal(W[r], oracle.xi_words(seed, t, j, q))
+        # neighbouring windows tile without overlap or gap
+        assert np.array_equal(oracle.xi_words_range(seed, t, j, q0 + 3, q0 + nq), W[3:])
+
+
+def test_box_muller_many_is_box_muller_row_by_row():
+    rng = np.random.default_rng(99)
+    words = rng.integers(0, 1 << 32, size=(400, 4), dtype=np.uint64).astype(np.uint32)
+    words[0] = [0, 0, MASK, MASK]                       # extremes of radius and angle
+    words[1] = [MASK, 0x40000000, 0x200, 0x80000000]
+    Z = oracle.box_muller_many(words)
+    assert Z.shape == (400, 4) and Z.dtype == np.float64
+    two_pi = 2 * math.pi
+    for r in range(400):
+        assert np.array_equal(Z[r], oracle.box_muller(words[r]))
+        # and against the closed form itself, written with the math module
+        for pair in range(2):
+            u1 = ((int(words[r, 2 * pair]) >> 9) + 0.5) / 2**23
+            u2 = ((int(words[r, 2 * pair + 1]) >> 9) + 0.5) / 2**23
+            rad = math.sqrt(-2.0 * math.log(u1))
+            assert math.isclose(Z[r, 2 * pair], rad * math.cos(two_pi * u2), rel_tol=1e-12, abs_tol=1e-13)
+            assert math.isclose(Z[r, 2 * pair + 1], rad * math.sin(two_pi * u2), rel_tol=1e-12, abs_tol=1e-13)
+    # rows are independent of their neighbours: a permutation of the rows permutes the output
+    perm = rng.permutation(400)
+    assert np.array_equal(oracle.box_muller_many(words[perm]), Z[perm])
