@@ -25,7 +25,13 @@
  *   - Work is enqueued on the context's stream (core_set_stream; default: the
  *     legacy default stream) and the call returns without synchronising,
  *     except the *_host entry points, which return after their last copy has
- *     completed, and any call that has to grow the workspace (cudaMalloc).
+ *     completed (also when they fail half-way: no copy is still reading or
+ *     writing the caller's buffers after the return), and any call that has to
+ *     grow the workspace: core_project, core_round, core_round_host and the
+ *     least-squares steps free and re-allocate it (cudaFree / cudaMalloc, which
+ *     synchronise the device) when the one they hold is too small.  A caller
+ *     that must not meet that synchronisation later takes it up front with
+ *     core_reserve_workspace.
  *   - Return value: CORE_OK or a negative error code.  A failing call launches
  *     nothing for CORE_EINVAL; outputs are unspecified after any error, but no
  *     call writes outside the extents stated here.  Nothing prints or aborts.
@@ -79,6 +85,14 @@ uint32_t core_get_round(const core_ctx *ctx);
 /* Bytes of device workspace the context currently holds. */
 size_t core_workspace_bytes(const core_ctx *ctx);
 
+/*
+ * Grow the workspace now to what core_project and core_round need for n machines of the given
+ * dtype (the context's d and m), so that those calls find it large enough and neither allocate
+ * nor synchronise.  May synchronise the device itself.  CORE_ENOMEM leaves the context usable
+ * (with no workspace; the next call tries again).
+ */
+int core_reserve_workspace(core_ctx *ctx, int32_t n, int dtype);
+
 const char *core_strerror(int code);
 int core_last_cuda_error(const core_ctx *ctx);
 
@@ -86,7 +100,8 @@ int core_last_cuda_error(const core_ctx *ctx);
  * Device-side status.  The tensor-memory projection kernel hands buffers between
  * its warps with barriers whose waits are bounded; a wait that runs out makes
  * the kernel finish early (its output is then meaningless) and records a
- * non-zero code in a per-device status word.  This call synchronises the
+ * non-zero code in a per-device status word.  A wait gives up after 100 ms of
+ * the device's global timer; waits that are served take microseconds.  This call synchronises the
  * current device, stores the word in *status_out (host pointer; 0 = every wait
  * was served) and clears it.  Not part of the paper: run-time diagnostics.
  */
@@ -154,8 +169,8 @@ int core_round_host(core_ctx *ctx, const void *G_host, int dtype, int32_t n, int
  * synchronisation is not allowed.  core_init and core_project obtain a workspace with
  * cudaMalloc; this call takes no context and obtains nothing.  The per-CTA partial sums of
  * the projection go to a fixed array of CORE_STATIC_SCRATCH_FLOATS floats (4 MiB) that is
- * part of the library image: every GPU that loads the library holds it until the process
- * exits.
+ * part of the library image: every GPU onto which the library's code has been loaded holds it
+ * until the process exits.
  *
  * Computes P[i*m + j] = <g_i, xi_j> exactly as core_project does for the generator keyed by
  * (seed, round t); arguments as for core_project, plus d, m, seed and t passed directly.
@@ -168,8 +183,15 @@ int core_round_host(core_ctx *ctx, const void *G_host, int dtype, int32_t n, int
  * used: slower, and the result may differ from core_project's in the last bits (same bound
  * against the exact value).
  *
- * The first call on a device looks up the array's device address (no allocation, no
- * synchronisation of the device); make that first call outside any stream capture.
+ * The first call on a device is a set-up call: it looks up the array's device address, and with
+ * CUDA's default lazy module loading that is also when the driver loads this part of the library
+ * onto the device and reserves the 4 MiB (the kernels are loaded at their first launch likewise).
+ * So the first call per device can itself need device memory, and can fail with CORE_ECUDA on a
+ * device that is already full: make it early, before the application claims the device, and
+ * outside any stream capture.  Later calls allocate nothing.  (With CUDA_MODULE_LOADING=EAGER in
+ * the environment the cost moves to the moment the library is loaded.)
+ * G_dev and P_dev must belong to the current device (checked; CORE_EINVAL otherwise): the scratch
+ * array used is the current device's.
  * All calls share the one array, which keeps the previous call's contents: nothing in it
  * needs to start at zero (every entry is written before it is read within a call), but two
  * calls whose kernels overlap on the GPU -- different streams, no dependency between them --
@@ -225,11 +247,38 @@ int core_agd_step(core_ctx *ctx, core_ls *ls, float h, float beta, float *x_dev,
 int core_gd_step_guarded(core_ctx *ctx, core_ls *ls, float h, float *x_dev, double *f_dev,
                          int32_t *accepted_dev);
 
-/* loss_dev[0] = f(x) as a double, computed on the device. */
+/*
+ * f(x) as a double, computed on the device in a fixed order (the objective of Algorithm 2's
+ * least-squares instance).  core_ls_loss leaves it in loss_dev[0] (DEVICE pointer: the guarded step
+ * consumes it there without a host round trip); core_ls_loss_host also enqueues its copy to
+ * loss_host[0] (HOST pointer, pinned for an asynchronous copy) on the context's stream: read it
+ * after synchronising that stream.  Neither call synchronises.
+ */
 int core_ls_loss(core_ctx *ctx, core_ls *ls, const float *x_dev, double *loss_dev);
+int core_ls_loss_host(core_ctx *ctx, core_ls *ls, const float *x_dev, double *loss_host);
 
 /* G_out_dev[i*d + k] = g_i[k] at x (the machine gradients alone; n*d floats). */
 int core_ls_gradients(core_ctx *ctx, core_ls *ls, const float *x_dev, float *G_out_dev);
+
+/* ---- failure paths, made on the host or bounded on the device (no counterpart in the paper) ---- */
+
+/*
+ * The next `count` device allocations of this library fail as if the device were out of memory
+ * (count = 0 switches this off).  Lets a test see CORE_ENOMEM from core_init, core_project,
+ * core_round_host, core_ls_create ... without exhausting a GPU: a failing call launches nothing and
+ * leaves its context usable.
+ */
+int core_debug_fail_allocations(int count);
+
+/*
+ * Runs one small CTA whose first warp waits, with the bounded-wait helper of the tensor-memory
+ * projection, on a barrier that nobody completes; after limit_us microseconds (1..100000) the wait
+ * gives up, the device status word receives `code` (>= 1; read and clear it with
+ * core_device_status) and the kernel returns by its normal exit.  observed_host[0] = 0 if the wait
+ * ran out (1 if it was served, which cannot happen), observed_host[1] = 1 if the CTA's second warp
+ * saw the abort flag.  Synchronises.  Uses no tensor-core instruction.
+ */
+int core_debug_wait_timeout(uint32_t limit_us, int32_t code, uint32_t observed_host[2]);
 
 /* ---- generator windows (for checking the generator itself) ------------------- */
 
@@ -249,6 +298,25 @@ int core_debug_box_muller(core_ctx *ctx, const uint32_t *words_dev, int64_t nb, 
  * tiles of d, dynamic shared memory bytes.
  */
 int core_debug_project_plan(int32_t n, int32_t m, int64_t d, int dtype, int32_t sm_count, int64_t out[10]);
+
+/*
+ * Instruction-rate probes (no counterpart in the paper: they support the roofline of the round kernels,
+ * which are bound by instruction issue).  Kind k < core_debug_pipe_kinds() - 3 runs a loop whose body
+ * is counts_out[0..6] = (32x32->64-bit multiplies, fp32 multiply-adds, packed fp32 multiply-adds,
+ * three-input logic ops, special-function calls, fp64 multiply-adds, 32-bit integer multiply-adds),
+ * all on independent chains (core_debug_pipe_mix reports the counts, all zero for the last three
+ * kinds).  The last three kinds run rounds 2..9 of Philox for four counters per body with the wide
+ * multiply done by the integer multiplier, by the fp64 unit plus a 32-bit multiply, or half and half;
+ * their checksums must agree (same words).
+ * core_debug_pipe_cycles launches the loop on every SM with warps_per_scheduler (2, 4 or 8) warps
+ * resident per scheduler, synchronises, and stores in *cycles_per_body_out (host pointer) the SM cycles
+ * one scheduler spends per loop body and warp, and in *checksum_out (host pointer, may be NULL) a
+ * digest of the loop results.  Allocates and frees its own small device buffers.
+ */
+int core_debug_pipe_kinds(void);
+int core_debug_pipe_mix(int kind, int32_t counts_out[7]);
+int core_debug_pipe_cycles(int kind, int warps_per_scheduler, int iters, uint32_t seed, double *cycles_per_body_out,
+                           uint32_t *checksum_out);
 
 #ifdef __cplusplus
 }

@@ -45,12 +45,20 @@ _SIGNATURES = {
     "core_gd_step_guarded": ([_c.c_void_p, _c.c_void_p, _c.c_float, _c.c_void_p, _c.c_void_p, _c.c_void_p],
                              _c.c_int),
     "core_ls_loss": ([_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p], _c.c_int),
+    "core_ls_loss_host": ([_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p], _c.c_int),
+    "core_reserve_workspace": ([_c.c_void_p, _c.c_int32, _c.c_int], _c.c_int),
+    "core_debug_fail_allocations": ([_c.c_int], _c.c_int),
+    "core_debug_wait_timeout": ([_c.c_uint32, _c.c_int32, _c.POINTER(_c.c_uint32)], _c.c_int),
     "core_ls_gradients": ([_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p], _c.c_int),
     "core_debug_philox": ([_c.c_void_p, _c.c_uint32, _c.c_uint64, _c.c_int64, _c.c_void_p], _c.c_int),
     "core_debug_gaussians": ([_c.c_void_p, _c.c_uint32, _c.c_uint64, _c.c_int64, _c.c_void_p], _c.c_int),
     "core_debug_box_muller": ([_c.c_void_p, _c.c_void_p, _c.c_int64, _c.c_void_p], _c.c_int),
     "core_project_static": ([_c.c_uint64, _c.c_uint32, _c.c_int64, _c.c_int32, _c.c_void_p, _c.c_int, _c.c_int32,
                              _c.c_int64, _c.c_void_p, _c.c_void_p, _c.POINTER(_c.c_int)], _c.c_int),
+    "core_debug_pipe_kinds": ([], _c.c_int),
+    "core_debug_pipe_mix": ([_c.c_int, _c.POINTER(_c.c_int32)], _c.c_int),
+    "core_debug_pipe_cycles": ([_c.c_int, _c.c_int, _c.c_int, _c.c_uint32, _c.POINTER(_c.c_double),
+                                _c.POINTER(_c.c_uint32)], _c.c_int),
     "core_debug_project_plan": ([_c.c_int32, _c.c_int32, _c.c_int64, _c.c_int, _c.c_int32,
                                  _c.POINTER(_c.c_int64)], _c.c_int),
 }
@@ -124,6 +132,43 @@ def core_debug_project_plan(n: int, m: int, d: int, dtype: int = CORE_F32, sm_co
     return dict(zip(keys, (int(v) for v in out)))
 
 
+def core_debug_pipe_kinds() -> int:
+    return int(lib().core_debug_pipe_kinds())
+
+
+def core_debug_pipe_mix(kind: int) -> tuple:
+    out = (ctypes.c_int32 * 7)()
+    rc = lib().core_debug_pipe_mix(kind, out)
+    if rc != CORE_OK:
+        raise CoreError(rc, "core_debug_pipe_mix")
+    return tuple(int(v) for v in out)
+
+
+def core_debug_pipe_cycles(kind: int, warps_per_scheduler: int = 4, iters: int = 2048, seed: int = 1):
+    """(SM cycles a scheduler spends per loop body and warp, checksum of the loop results)."""
+    cyc, chk = ctypes.c_double(0.0), ctypes.c_uint32(0)
+    rc = lib().core_debug_pipe_cycles(kind, warps_per_scheduler, iters, seed, ctypes.byref(cyc), ctypes.byref(chk))
+    if rc != CORE_OK:
+        raise CoreError(rc, "core_debug_pipe_cycles")
+    return float(cyc.value), int(chk.value)
+
+
+def core_debug_fail_allocations(count: int) -> None:
+    """The next `count` device allocations of the library fail (0 switches this off)."""
+    rc = lib().core_debug_fail_allocations(int(count))
+    if rc != CORE_OK:
+        raise CoreError(rc, "core_debug_fail_allocations")
+
+
+def core_debug_wait_timeout(limit_us: int, code: int) -> tuple:
+    """(wait was served, second warp saw the abort flag) of the bounded-wait test kernel."""
+    out = (ctypes.c_uint32 * 2)()
+    rc = lib().core_debug_wait_timeout(int(limit_us), int(code), out)
+    if rc != CORE_OK:
+        raise CoreError(rc, "core_debug_wait_timeout")
+    return int(out[0]), int(out[1])
+
+
 def core_device_status() -> int:
     """Synchronises the current device; returns and clears the status word that a kernel raises
     when one of its bounded waits runs out (0: every wait was served)."""
@@ -191,6 +236,9 @@ class Core:
 
     def core_workspace_bytes(self) -> int:
         return int(lib().core_workspace_bytes(self._h))
+
+    def core_reserve_workspace(self, n: int, dtype: int = CORE_F32):
+        self._check(lib().core_reserve_workspace(self._h, int(n), int(dtype)), "core_reserve_workspace")
 
     # -- the round ------------------------------------------------------------------
     def core_project(self, G_dev: torch.Tensor, P_dev: torch.Tensor | None = None) -> torch.Tensor:
@@ -267,6 +315,13 @@ class Core:
         self._check(lib().core_ls_loss(self._h, ls._h, _dev(x_dev, torch.float32, self.d),
                                        _dev(loss_dev, torch.float64, 1)), "core_ls_loss")
         return loss_dev
+
+    def core_ls_loss_host(self, ls: "LeastSquares", x_dev: torch.Tensor, loss_host: torch.Tensor):
+        if loss_host.is_cuda or loss_host.dtype != torch.float64 or loss_host.numel() < 1:
+            raise ValueError("loss_host must be a host float64 tensor")
+        self._check(lib().core_ls_loss_host(self._h, ls._h, _dev(x_dev, torch.float32, self.d), loss_host.data_ptr()),
+                    "core_ls_loss_host")
+        return loss_host
 
     def core_ls_gradients(self, ls: "LeastSquares", x_dev: torch.Tensor, G_out_dev: torch.Tensor | None = None):
         if G_out_dev is None:

@@ -2,6 +2,7 @@
 // Every entry point is declared, with its contract, in include/core.h.
 #include "core.h"
 
+#include <atomic>
 #include <new>
 
 #include "core_internal.h"
@@ -60,6 +61,21 @@ int cuda_fail(core_ctx *ctx, cudaError_t e) {
         if (e__ != cudaSuccess) return cuda_fail((ctx), e__); \
     } while (0)
 
+// Every device allocation of the library goes through here, so that tests can make the next ones fail
+// on the host (core_debug_fail_allocations) and see the out-of-memory paths without exhausting a GPU.
+std::atomic<int> g_fail_allocations{0};
+
+cudaError_t core_malloc(void **out, size_t bytes) {
+    int left = g_fail_allocations.load();
+    while (left > 0) {
+        if (g_fail_allocations.compare_exchange_weak(left, left - 1)) {
+            *out = nullptr;
+            return cudaErrorMemoryAllocation;
+        }
+    }
+    return cudaMalloc(out, bytes);
+}
+
 bool on_device(int device) {
     int cur = -1;
     return cudaGetDevice(&cur) == cudaSuccess && cur == device;
@@ -74,7 +90,7 @@ int ensure_workspace(core_ctx *ctx, size_t bytes) {
         if (e != cudaSuccess) return cuda_fail(ctx, e);
     }
     bytes = round_up(bytes, (size_t)1 << 20);
-    cudaError_t e = cudaMalloc(&ctx->ws, bytes);
+    cudaError_t e = core_malloc(&ctx->ws, bytes);
     if (e != cudaSuccess) {
         ctx->ws = nullptr;
         cudaGetLastError();
@@ -147,7 +163,7 @@ int core_init(core_ctx **out, uint64_t seed, int64_t d, int32_t m) {
     ctx->slab_bytes = 0;
     cudaError_t e = cudaGetDevice(&ctx->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
-    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->pbar), (size_t)m * sizeof(float));
+    if (e == cudaSuccess) e = core_malloc(reinterpret_cast<void **>(&ctx->pbar), (size_t)m * sizeof(float));
     if (e != cudaSuccess) {
         cudaGetLastError();
         const int rc = e == cudaErrorMemoryAllocation ? CORE_ENOMEM : CORE_ECUDA;
@@ -228,6 +244,15 @@ int core_project(core_ctx *ctx, const void *G_dev, int dtype, int32_t n, int64_t
                         ctx->stream);
 }
 
+int core_reserve_workspace(core_ctx *ctx, int32_t n, int dtype) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (n < 1 || !valid_dtype(dtype)) return CORE_EINVAL;
+    // what core_round needs (partial sums + the messages); core_project needs the first part only
+    const size_t pb = partial_bytes(ctx, n, ctx->d, dtype);
+    const size_t Pb = round_up((size_t)n * ctx->m * sizeof(float), 256);
+    return ensure_workspace(ctx, pb + Pb);
+}
+
 int core_aggregate(core_ctx *ctx, const float *P_dev, int32_t n, float *pbar_dev) {
     if (int rc = check_ctx(ctx)) return rc;
     if (!P_dev || !pbar_dev || n < 1) return CORE_EINVAL;
@@ -275,18 +300,46 @@ int core_round(core_ctx *ctx, const void *G_dev, int dtype, int32_t n, int64_t l
     return round_with_epilogue(ctx, G_dev, dtype, n, ldg, pbar_dev, gtilde_dev, nullptr);
 }
 
+static int round_host_body(core_ctx *ctx, const void *G_host, int dtype, int32_t n, int64_t ldg, float *pbar_host,
+                           float *gtilde_host);
+
 int core_round_host(core_ctx *ctx, const void *G_host, int dtype, int32_t n, int64_t ldg, float *pbar_host,
                     float *gtilde_host) {
     if (int rc = check_ctx(ctx)) return rc;
     if (!G_host || !pbar_host || !gtilde_host || n < 1 || ldg < ctx->d || !valid_dtype(dtype)) return CORE_EINVAL;
+    const int rc = round_host_body(ctx, G_host, dtype, n, ldg, pbar_host, gtilde_host);
+    if (rc != CORE_OK && ctx->host_ready) {
+        // copies enqueued before the failure may still be reading G_host or writing the outputs: the
+        // caller gets its buffers back only once both streams have drained (a second error is ignored)
+        const int first = ctx->last_cuda;
+        cudaStreamSynchronize(ctx->work_stream);
+        cudaStreamSynchronize(ctx->copy_stream);
+        cudaGetLastError();
+        ctx->last_cuda = first;
+    }
+    return rc;
+}
+
+static int round_host_body(core_ctx *ctx, const void *G_host, int dtype, int32_t n, int64_t ldg, float *pbar_host,
+                           float *gtilde_host) {
     if (!ctx->host_ready) {
-        CORE_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
-        CORE_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->work_stream, cudaStreamNonBlocking));
-        for (int s = 0; s < 2; ++s) {
-            CORE_CUDA(ctx, cudaEventCreateWithFlags(&ctx->in_ready[s], cudaEventDisableTiming));
-            CORE_CUDA(ctx, cudaEventCreateWithFlags(&ctx->in_free[s], cudaEventDisableTiming));
-            CORE_CUDA(ctx, cudaEventCreateWithFlags(&ctx->out_ready[s], cudaEventDisableTiming));
-            CORE_CUDA(ctx, cudaEventCreateWithFlags(&ctx->out_free[s], cudaEventDisableTiming));
+        // all or nothing: a half-made set of streams and events is torn down again
+        cudaError_t e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        e = cudaStreamCreateWithFlags(&ctx->work_stream, cudaStreamNonBlocking);
+        if (e != cudaSuccess) {
+            cudaStreamDestroy(ctx->copy_stream);
+            return cuda_fail(ctx, e);
+        }
+        cudaEvent_t *events[8] = {&ctx->in_ready[0], &ctx->in_ready[1], &ctx->in_free[0], &ctx->in_free[1],
+                                  &ctx->out_ready[0], &ctx->out_ready[1], &ctx->out_free[0], &ctx->out_free[1]};
+        int made = 0;
+        for (; made < 8 && e == cudaSuccess; ++made) e = cudaEventCreateWithFlags(events[made], cudaEventDisableTiming);
+        if (e != cudaSuccess) {
+            for (int k = 0; k + 1 < made; ++k) cudaEventDestroy(*events[k]);
+            cudaStreamDestroy(ctx->copy_stream);
+            cudaStreamDestroy(ctx->work_stream);
+            return cuda_fail(ctx, e);
         }
         ctx->host_ready = true;
     }
@@ -306,7 +359,7 @@ int core_round_host(core_ctx *ctx, const void *G_host, int dtype, int32_t n, int
             ctx->slab = nullptr;
             ctx->slab_bytes = 0;
         }
-        cudaError_t e = cudaMalloc(&ctx->slab, need_slab);
+        cudaError_t e = core_malloc(&ctx->slab, need_slab);
         if (e != cudaSuccess) {
             cudaGetLastError();
             ctx->last_cuda = (int)e;
@@ -397,7 +450,7 @@ int core_ls_create(core_ls **out, const float *A_dev, const float *b_dev, int32_
     const size_t gt_b = round_up((size_t)d * sizeof(float), 256);
     const size_t scalars_b = 256;                          // trial loss (double) and acceptance flag
     char *base = nullptr;
-    e = cudaMalloc(reinterpret_cast<void **>(&base), res_b + part_b + G_b + gt_b + scalars_b);
+    e = core_malloc(reinterpret_cast<void **>(&base), res_b + part_b + G_b + gt_b + scalars_b);
     if (e != cudaSuccess) {
         cudaGetLastError();
         delete ls;
@@ -501,6 +554,41 @@ int core_ls_loss(core_ctx *ctx, core_ls *ls, const float *x_dev, double *loss_de
     if (!ls || !x_dev || !loss_dev || ls->d != ctx->d || ls->device != ctx->device) return CORE_EINVAL;
     CORE_CUDA(ctx, launch_ls_residual(ls->A, ls->b, x_dev, ls->n, ls->rows, ls->d, ls->res, ctx->stream));
     CORE_CUDA(ctx, launch_ls_loss(ls->res, ls->n, ls->rows, loss_dev, ctx->stream));
+    return CORE_OK;
+}
+
+int core_ls_loss_host(core_ctx *ctx, core_ls *ls, const float *x_dev, double *loss_host) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!ls || !x_dev || !loss_host || ls->d != ctx->d || ls->device != ctx->device) return CORE_EINVAL;
+    CORE_CUDA(ctx, launch_ls_residual(ls->A, ls->b, x_dev, ls->n, ls->rows, ls->d, ls->res, ctx->stream));
+    CORE_CUDA(ctx, launch_ls_loss(ls->res, ls->n, ls->rows, ls->f_trial, ctx->stream));
+    CORE_CUDA(ctx, cudaMemcpyAsync(loss_host, ls->f_trial, sizeof(double), cudaMemcpyDeviceToHost, ctx->stream));
+    return CORE_OK;
+}
+
+/* ---- run-time diagnostics ------------------------------------------------------ */
+
+int core_debug_fail_allocations(int count) {
+    if (count < 0) return CORE_EINVAL;
+    g_fail_allocations.store(count);
+    return CORE_OK;
+}
+
+int core_debug_wait_timeout(uint32_t limit_us, int32_t code, uint32_t observed_host[2]) {
+    if (!observed_host || limit_us < 1 || limit_us > 100000 || code < 1) return CORE_EINVAL;
+    uint32_t *observed = nullptr;
+    if (core_malloc(reinterpret_cast<void **>(&observed), 2 * sizeof(uint32_t)) != cudaSuccess) {
+        cudaGetLastError();
+        return CORE_ENOMEM;
+    }
+    cudaError_t e = cudaMemset(observed, 0xFF, 2 * sizeof(uint32_t));
+    if (e == cudaSuccess) e = launch_wait_timeout_probe((uint64_t)limit_us * 1000ull, code, observed, nullptr);
+    if (e == cudaSuccess) e = cudaMemcpy(observed_host, observed, 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost);
+    cudaFree(observed);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return CORE_ECUDA;
+    }
     return CORE_OK;
 }
 

@@ -46,6 +46,10 @@ cudaError_t launch_project_tc(const ProjectPlan &plan, const RoundKeys &keys, ui
                               int dtype, int32_t n, int64_t ldg, int64_t d, int32_t m, uint64_t q_base,
                               float *partial, cudaStream_t stream);
 cudaError_t project_tc_take_status(int *status);
+// One small CTA that waits, with the projection's bounded-wait helper, on a barrier nobody completes:
+// after limit_ns the wait gives up, the status word receives `code`, and observed_dev[0..1] (device)
+// become {0: the wait did not succeed, 1: the second warp saw the abort flag}.
+cudaError_t launch_wait_timeout_probe(uint64_t limit_ns, int code, uint32_t *observed_dev, cudaStream_t stream);
 
 // One projection pass over coordinates [0, d) of rows G + i*ldg, i < n <= 16.
 // q_base is the global index of the block holding coordinate 0 of G (non-zero when G

@@ -1,0 +1,333 @@
+// Instruction-rate probes (test-only entry point core_debug_pipe_cycles).
+//
+// The round kernels are bound by instruction issue, so their roofline rests on how many cycles of a
+// scheduler each instruction class costs on this GPU.  The probes here measure that directly: every
+// warp runs a loop whose body is a fixed mix of independent dependent-chains (wide integer multiplies,
+// fp32 and packed fp32 multiply-adds, three-input logic, special-function calls, fp64 multiply-adds,
+// 32-bit integer multiply-adds), and reports the SM cycles it took; with W warps resident per scheduler
+// the scheduler's cost of one loop body is cycles / (iterations * W).  Cycle counts do not depend on the
+// clock frequency.  Two further probes run the Philox rounds of the generator alone, with the 32x32->64
+// multiply done by the integer multiplier or by the fp64 unit (see philox_probe_kernel).
+#include "core.h"
+
+#include <vector>
+
+#include "core_internal.h"
+
+using namespace core;
+
+namespace {
+
+struct Mix {
+    int wide, ffma, ffma2, lop3, mufu, dfma, imad;
+};
+
+// Loop bodies on offer: index = `kind` of core_debug_pipe_cycles.
+constexpr Mix kMixes[] = {
+    {16, 0, 0, 0, 0, 0, 0},    //  0  wide multiply alone
+    {0, 64, 0, 0, 0, 0, 0},    //  1  fp32 multiply-add
+    {0, 0, 32, 0, 0, 0, 0},    //  2  packed fp32 multiply-add (two lanes per instruction)
+    {0, 0, 0, 64, 0, 0, 0},    //  3  three-input logic
+    {0, 0, 0, 0, 16, 0, 0},    //  4  special function (log2)
+    {0, 0, 0, 0, 0, 32, 0},    //  5  fp64 multiply-add
+    {0, 0, 0, 0, 0, 0, 32},    //  6  32-bit integer multiply-add
+    {16, 16, 0, 0, 0, 0, 0},   //  7  wide + fp32
+    {16, 32, 0, 0, 0, 0, 0},   //  8
+    {16, 64, 0, 0, 0, 0, 0},   //  9
+    {16, 0, 16, 0, 0, 0, 0},   // 10  wide + packed fp32
+    {16, 0, 0, 32, 0, 0, 0},   // 11  wide + logic
+    {16, 32, 0, 32, 0, 0, 0},  // 12  wide + fp32 + logic
+    {16, 0, 0, 0, 0, 16, 0},   // 13  wide + fp64
+    {0, 0, 0, 0, 0, 16, 16},   // 14  fp64 + 32-bit integer multiply-add
+    {8, 0, 0, 0, 0, 8, 8},     // 15  wide + fp64 + integer
+    {0, 32, 0, 0, 0, 16, 16},  // 16  fp64 + integer + fp32
+    {0, 0, 0, 18, 0, 16, 16},  // 17  fp64 + integer + logic (the Philox mix with the fp64 high word)
+    {16, 0, 0, 18, 0, 0, 0},   // 18  wide + logic (the Philox mix)
+    {0, 0, 0, 0, 8, 0, 0},     // 19  special function, half as many
+    {16, 0, 0, 0, 8, 0, 0},    // 20  wide + special function
+};
+constexpr int kMixCount = sizeof(kMixes) / sizeof(kMixes[0]);
+constexpr int kPhiloxKinds = 3;   // kinds kMixCount .. kMixCount+2: the Philox probes
+
+__device__ __forceinline__ unsigned long long mad_wide(uint32_t a, uint32_t b, unsigned long long c) {
+    unsigned long long d;
+    asm volatile("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ float ffma_v(float a, float b, float c) {
+    float d;
+    asm volatile("fma.rn.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long ffma2_v(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm volatile("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t lop3_v(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm volatile("lop3.b32 %0, %1, %2, %3, 0x6A;" : "=r"(d) : "r"(a), "r"(b), "r"(c));   // (a & b) ^ c
+    return d;
+}
+__device__ __forceinline__ float lg2_v(float a) {
+    float d;
+    asm volatile("lg2.approx.ftz.f32 %0, %1;" : "=f"(d) : "f"(a));
+    return d;
+}
+__device__ __forceinline__ double dfma_v(double a, double b, double c) {
+    double d;
+    asm volatile("fma.rz.f64 %0, %1, %2, %3;" : "=d"(d) : "d"(a), "d"(b), "d"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t imad_v(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm volatile("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
+template <int N>
+struct Chains {
+    static constexpr int value = N == 0 ? 1 : (N < 8 ? N : 8);   // independent chains per class
+};
+
+// One warp's loop: `iters` bodies of the mix, every class on its own independent chains.
+template <int KIND>
+__global__ void __launch_bounds__(256)
+mix_probe_kernel(int iters, uint32_t seed, long long *cycles, uint32_t *sink) {
+    constexpr Mix M = kMixes[KIND];
+    constexpr int CW = Chains<M.wide>::value, CF = Chains<M.ffma>::value, CP = Chains<M.ffma2>::value,
+                  CL = Chains<M.lop3>::value, CM = Chains<M.mufu>::value, CD = Chains<M.dfma>::value,
+                  CI = Chains<M.imad>::value;
+    const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x;
+    unsigned long long w[CW];
+    float f[CF];
+    unsigned long long p[CP];
+    uint32_t l[CL];
+    float s[CM];
+    double d[CD];
+    uint32_t im[CI];
+    for (int c = 0; c < CW; ++c) w[c] = (unsigned long long)(tid * 2654435761u + seed + c) * 0x9E3779B97F4A7C15ull;
+    for (int c = 0; c < CF; ++c) f[c] = 1.0f + 1e-3f * (float)((tid + c) & 255);
+    for (int c = 0; c < CP; ++c) p[c] = ((unsigned long long)__float_as_uint(1.0f + 1e-3f * c) << 32) | __float_as_uint(0.5f + 1e-3f * (tid & 63));
+    for (int c = 0; c < CL; ++c) l[c] = tid * 747796405u + seed * (c + 1);
+    for (int c = 0; c < CM; ++c) s[c] = 1.5f + (float)((tid + c) & 31);
+    for (int c = 0; c < CD; ++c) d[c] = 1.0 + 1e-6 * (double)((tid + c) & 1023);
+    for (int c = 0; c < CI; ++c) im[c] = tid + seed + c;
+    const float fa = 0.999f + 1e-9f * (float)seed, fb = 1e-3f;
+    const unsigned long long pa = ((unsigned long long)__float_as_uint(fa) << 32) | __float_as_uint(fa);
+    const unsigned long long pb = ((unsigned long long)__float_as_uint(fb) << 32) | __float_as_uint(fb);
+    const double da = 0.9999990 + 1e-12 * (double)seed, db = 1e-7;
+    const uint32_t mult = 0xD2511F53u + 2u * seed;
+
+    __syncthreads();
+    const long long t0 = clock64();
+    for (int it = 0; it < iters; ++it) {
+        constexpr int LONGEST = M.wide > M.ffma ? M.wide : M.ffma;
+        constexpr int L2 = M.ffma2 > M.lop3 ? M.ffma2 : M.lop3;
+        constexpr int L3 = M.mufu > M.dfma ? M.mufu : M.dfma;
+        constexpr int L4 = L2 > L3 ? L2 : L3;
+        constexpr int L5 = LONGEST > L4 ? LONGEST : L4;
+        constexpr int STEPS = L5 > M.imad ? L5 : M.imad;
+        // emit the classes interleaved in proportion to their counts
+#pragma unroll
+        for (int st = 0; st < STEPS; ++st) {
+            if ((st + 1) * M.wide / STEPS > st * M.wide / STEPS) {
+                const int c = (st * M.wide / STEPS) % CW;
+                w[c] = mad_wide((uint32_t)w[c], mult, w[c]);
+            }
+            if ((st + 1) * M.dfma / STEPS > st * M.dfma / STEPS) {
+                const int c = (st * M.dfma / STEPS) % CD;
+                d[c] = dfma_v(d[c], da, db);
+            }
+            if ((st + 1) * M.imad / STEPS > st * M.imad / STEPS) {
+                const int c = (st * M.imad / STEPS) % CI;
+                im[c] = imad_v(im[c], mult, im[(c + 1) % CI]);
+            }
+            if ((st + 1) * M.ffma / STEPS > st * M.ffma / STEPS) {
+                const int c = (st * M.ffma / STEPS) % CF;
+                f[c] = ffma_v(f[c], fa, fb);
+            }
+            if ((st + 1) * M.ffma2 / STEPS > st * M.ffma2 / STEPS) {
+                const int c = (st * M.ffma2 / STEPS) % CP;
+                p[c] = ffma2_v(p[c], pa, pb);
+            }
+            if ((st + 1) * M.lop3 / STEPS > st * M.lop3 / STEPS) {
+                const int c = (st * M.lop3 / STEPS) % CL;
+                l[c] = lop3_v(l[c], l[(c + 1) % CL], mult);
+            }
+            if ((st + 1) * M.mufu / STEPS > st * M.mufu / STEPS) {
+                const int c = (st * M.mufu / STEPS) % CM;
+                s[c] = lg2_v(s[c]);
+            }
+        }
+    }
+    const long long t1 = clock64();
+    uint32_t acc = 0;
+    for (int c = 0; c < CW; ++c) acc ^= (uint32_t)w[c] ^ (uint32_t)(w[c] >> 32);
+    for (int c = 0; c < CF; ++c) acc ^= __float_as_uint(f[c]);
+    for (int c = 0; c < CP; ++c) acc ^= (uint32_t)p[c] ^ (uint32_t)(p[c] >> 32);
+    for (int c = 0; c < CL; ++c) acc ^= l[c];
+    for (int c = 0; c < CM; ++c) acc ^= __float_as_uint(s[c]);
+    for (int c = 0; c < CD; ++c) acc ^= (uint32_t)__double2loint(d[c]) ^ (uint32_t)__double2hiint(d[c]);
+    for (int c = 0; c < CI; ++c) acc ^= im[c];
+    sink[tid] = acc;
+    if ((threadIdx.x & 31) == 0) cycles[tid >> 5] = t1 - t0;
+}
+
+// ---- Philox alone, with the 32x32 -> 64-bit multiply done three ways -----------------------------
+// MODE 0: the integer multiplier (mul.wide.u32), as the round kernels do.
+// MODE 1: high word from the fp64 unit, low word from a 32-bit integer multiply.  With
+//         a = 2^52 + x (x inserted as the low mantissa word of 2^52), fma.rz(a, M, 2^84 - 2^52 M)
+//         = 2^84 + x M rounded towards zero to a multiple of 2^32 (the spacing of doubles in
+//         [2^84, 2^85)), so the low mantissa word of the result is floor(x M / 2^32), exactly.
+// MODE 2: the multiply of counter word 0 as in mode 0, that of counter word 2 as in mode 1.
+template <int MODE>
+__device__ __forceinline__ void mul_hi_lo(uint32_t mult, double mult_d, double bias_d, uint32_t x, uint32_t &hi, uint32_t &lo) {
+    if constexpr (MODE == 0) {
+        mul_wide(mult, x, hi, lo);
+    } else {
+        const double a = __hiloint2double(0x43300000, (int)x);
+        double r;
+        asm("fma.rz.f64 %0, %1, %2, %3;" : "=d"(r) : "d"(a), "d"(mult_d), "d"(bias_d));
+        hi = (uint32_t)__double2loint(r);
+        lo = x * mult;
+    }
+}
+
+template <int MODE>
+__device__ __forceinline__ uint4 philox_tail(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, const RoundKeys &k,
+                                             double ma_d, double ba_d, double mb_d, double bb_d) {
+#pragma unroll
+    for (int r = 2; r < 10; ++r) {
+        uint32_t hi_a, lo_a, hi_b, lo_b;
+        mul_hi_lo<MODE == 2 ? 0 : MODE>(kPhiloxMulA, ma_d, ba_d, c0, hi_a, lo_a);
+        mul_hi_lo<MODE == 2 ? 1 : MODE>(kPhiloxMulB, mb_d, bb_d, c2, hi_b, lo_b);
+        c0 = hi_b ^ c1 ^ k.a[r];
+        c1 = lo_b;
+        c2 = hi_a ^ c3 ^ k.b[r];
+        c3 = lo_a;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+struct ProbeArgs {
+    RoundKeys keys;
+    int iters;
+    uint32_t seed;
+};
+
+// A warp's loop: four counters per iteration (four vectors, one coordinate block), rounds 2..9 of each.
+template <int MODE>
+__global__ void __launch_bounds__(256)
+philox_probe_kernel(const __grid_constant__ ProbeArgs a, long long *cycles, uint32_t *sink) {
+    const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x;
+    const double ma_d = (double)kPhiloxMulA, mb_d = (double)kPhiloxMulB;
+    const double two84 = 19342813113834066795298816.0, two52 = 4503599627370496.0;
+    const double ba_d = two84 - two52 * ma_d, bb_d = two84 - two52 * mb_d;       // exact: 32-bit integers times 2^52
+    JPart jp[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) jp[u] = philox_jpart(tid * 4 + u, 0, a.keys);
+    uint32_t acc0 = 0, acc1 = 0, acc2 = 0, acc3 = 0;
+    __syncthreads();
+    const long long t0 = clock64();
+    for (int it = 0; it < a.iters; ++it) {
+        const QPart qp = philox_qpart(a.seed + (uint32_t)it, 0, a.keys);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint4 w = philox_tail<MODE>(qp.hi_b ^ jp[u].x0, qp.lo_b, jp[u].x2 ^ qp.w3, jp[u].w3, a.keys, ma_d, ba_d,
+                                              mb_d, bb_d);
+            acc0 ^= w.x;
+            acc1 += w.y;
+            acc2 ^= w.z;
+            acc3 += w.w;
+        }
+    }
+    const long long t1 = clock64();
+    sink[tid] = acc0 ^ acc1 ^ acc2 ^ acc3;
+    if ((threadIdx.x & 31) == 0) cycles[tid >> 5] = t1 - t0;
+}
+
+template <int K = 0>
+cudaError_t launch_mix(int kind, int grid, int iters, uint32_t seed, long long *cycles, uint32_t *sink, cudaStream_t s) {
+    if constexpr (K < kMixCount) {
+        if (kind == K) {
+            mix_probe_kernel<K><<<grid, 256, 0, s>>>(iters, seed, cycles, sink);
+            return cudaGetLastError();
+        }
+        return launch_mix<K + 1>(kind, grid, iters, seed, cycles, sink, s);
+    } else {
+        return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+int core_debug_pipe_kinds(void) { return kMixCount + kPhiloxKinds; }
+
+int core_debug_pipe_mix(int kind, int32_t counts_out[7]) {
+    if (!counts_out || kind < 0 || kind >= kMixCount + kPhiloxKinds) return CORE_EINVAL;
+    Mix m{};
+    if (kind < kMixCount) m = kMixes[kind];
+    const int32_t v[7] = {m.wide, m.ffma, m.ffma2, m.lop3, m.mufu, m.dfma, m.imad};
+    for (int i = 0; i < 7; ++i) counts_out[i] = v[i];
+    return CORE_OK;
+}
+
+int core_debug_pipe_cycles(int kind, int warps_per_scheduler, int iters, uint32_t seed, double *cycles_per_body_out,
+                           uint32_t *checksum_out) {
+    if (!cycles_per_body_out || kind < 0 || kind >= kMixCount + kPhiloxKinds || iters < 1 || iters > (1 << 20) ||
+        (warps_per_scheduler != 2 && warps_per_scheduler != 4 && warps_per_scheduler != 8))
+        return CORE_EINVAL;
+    int device = 0, sm_count = 0;
+    if (cudaGetDevice(&device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
+        return CORE_ECUDA;
+    // 256-thread CTAs, all resident at once: warps_per_scheduler * 4 warps per SM
+    const int ctas_per_sm = warps_per_scheduler * 4 / 8;
+    const int grid = sm_count * ctas_per_sm;
+    const size_t warps = (size_t)grid * 8, threads = (size_t)grid * 256;
+    long long *cycles = nullptr;
+    uint32_t *sink = nullptr;
+    if (cudaMalloc(reinterpret_cast<void **>(&cycles), warps * sizeof(long long)) != cudaSuccess) return CORE_ENOMEM;
+    if (cudaMalloc(reinterpret_cast<void **>(&sink), threads * sizeof(uint32_t)) != cudaSuccess) {
+        cudaFree(cycles);
+        return CORE_ENOMEM;
+    }
+    cudaError_t e = cudaSuccess;
+    for (int rep = 0; rep < 2 && e == cudaSuccess; ++rep) {     // the first launch warms the instruction cache
+        if (kind < kMixCount) {
+            e = launch_mix(kind, grid, iters, seed, cycles, sink, nullptr);
+        } else {
+            ProbeArgs a{expand_keys(0x1234567ull + seed), iters, seed};
+            const int mode = kind - kMixCount;
+            if (mode == 0) philox_probe_kernel<0><<<grid, 256>>>(a, cycles, sink);
+            else if (mode == 1) philox_probe_kernel<1><<<grid, 256>>>(a, cycles, sink);
+            else philox_probe_kernel<2><<<grid, 256>>>(a, cycles, sink);
+            e = cudaGetLastError();
+        }
+        if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    }
+    std::vector<long long> host(warps);
+    std::vector<uint32_t> words(threads);
+    if (e == cudaSuccess) e = cudaMemcpy(host.data(), cycles, warps * sizeof(long long), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) e = cudaMemcpy(words.data(), sink, threads * sizeof(uint32_t), cudaMemcpyDeviceToHost);
+    cudaFree(cycles);
+    cudaFree(sink);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return CORE_ECUDA;
+    }
+    double sum = 0.0;
+    for (long long c : host) sum += (double)c;
+    *cycles_per_body_out = sum / (double)warps / (double)iters / (double)warps_per_scheduler;
+    if (checksum_out) {
+        uint32_t x = 0;
+        for (uint32_t v : words) x = x * 0x01000193u ^ v;
+        *checksum_out = x;
+    }
+    return CORE_OK;
+}
+
+}  // extern "C"

@@ -39,7 +39,7 @@ constexpr uint32_t kTcStageBytes = 2 * kTcPlaneA + 2 * kTcPlaneB;
 constexpr uint32_t kTcBarrierBytes = 128;
 constexpr uint32_t kTcSmemBytes = kTcStages * kTcStageBytes + kTcBarrierBytes + 1024;   // + alignment slack
 constexpr uint32_t kTcTmemColumns = 64;         // two buffers x (head products, tail products) x 16 columns
-constexpr uint32_t kTcSpinLimit = 1u << 22;
+constexpr uint64_t kTcWaitLimitNs = 100ull * 1000 * 1000;   // a wait gives up after 100 ms of the global timer
 
 __device__ int g_tc_status;                     // 0, or the code of a wait that ran out
 
@@ -78,10 +78,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: false when the phase did not complete within the limit.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t spin = 0; spin < kTcSpinLimit; ++spin)
-        if (mbar_try_wait(bar, parity)) return true;
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: false when the phase did not complete within limit_ns of the global timer (read only
+// once a first probe has failed, so a wait that is served at once costs one probe).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_t limit_ns = kTcWaitLimitNs) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    do {
+#pragma unroll 1
+        for (int probe = 0; probe < 64; ++probe)
+            if (mbar_try_wait(bar, parity)) return true;
+    } while (global_timer_ns() - t0 < limit_ns);
     return false;
 }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -254,17 +265,25 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
         atomicMax(&g_tc_status, code);
     };
     // Whole-warp wait.  The common case (the phase completed long ago) costs one probe and one vote.
+    // Has any warp of this CTA given up?  One answer for the whole warp: a flag raised between two lanes'
+    // reads must not split the warp (the lanes that stayed would wait for the ones that left).
+    auto aborted = [&]() { return __any_sync(0xffffffffu, *abort_flag != 0); };
+    // Whole-warp wait.  The common case (the phase completed long ago) costs one probe and one vote.
     auto warp_wait = [&](uint32_t bar, uint32_t parity, int code) {
         if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
-        bool ok = *abort_flag == 0 && mbar_wait(bar, parity);
-        ok = __all_sync(0xffffffffu, ok);
+        bool ok = !aborted();
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar, parity));
         if (!ok && lane == 0) give_up(code);
         return ok;
     };
     // One lane waits, patiently (the hardware may park it between probes).
     auto lane_wait = [&](uint32_t bar, uint32_t parity, int code) {
-        bool ok = false;
-        for (uint32_t spin = 0; spin < kTcSpinLimit && !ok; ++spin) ok = mbar_try_wait_patient(bar, parity, 2000u);
+        bool ok = mbar_try_wait(bar, parity);
+        if (!ok) {
+            const uint64_t t0 = global_timer_ns();
+            do ok = mbar_try_wait_patient(bar, parity, 2000u);
+            while (!ok && global_timer_ns() - t0 < kTcWaitLimitNs);
+        }
         if (!ok) give_up(code);
         return ok;
     };
@@ -407,7 +426,7 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
             // that no other warp can be issuing a later stage first.
             if (count > 0 && (uint32_t)warp == ((count - 1) & (kTcWarps - 1))) {
                 issue(prev_s, prev_ph, prev_st, prev_stages, prev_local);
-                if (*abort_flag) { alive = false; break; }
+                if (aborted()) { alive = false; break; }
             }
             fence_proxy_async_smem();                                // my stores, visible to the tensor core
             mbar_arrive(bar_full + 8 * s);
@@ -442,7 +461,47 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
     }
 }
 
+// Test kernel for the bounded waits: two warps share a barrier that expects one arrival nobody makes.
+// Warp 0 waits on it with the helper the projection uses (and a short limit), records the code when the
+// wait runs out and raises the CTA's abort flag; warp 1 watches the flag the way the projection's warps
+// do.  Both leave by the normal exit.  No tensor-core instruction, no tensor memory.
+__global__ void wait_timeout_probe_kernel(uint64_t limit_ns, int code, uint32_t *observed) {
+    __shared__ __align__(8) unsigned long long barrier_word;
+    __shared__ volatile uint32_t abort_flag;
+    const uint32_t bar = smem_u32(&barrier_word);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        abort_flag = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+    if (warp == 0) {
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(bar, 0, limit_ns));
+        if (!ok && lane == 0) {
+            abort_flag = 1;
+            atomicMax(&g_tc_status, code);
+        }
+        if (lane == 0) observed[0] = ok ? 1u : 0u;
+    } else {
+        // bounded too: at most ten times the limit
+        const uint64_t t0 = global_timer_ns();
+        bool seen = false;
+        for (;;) {                                                   // both votes are taken by the whole warp
+            seen = __any_sync(0xffffffffu, abort_flag != 0);
+            const bool time_up = __any_sync(0xffffffffu, global_timer_ns() - t0 >= 10 * limit_ns);
+            if (seen || time_up) break;
+        }
+        if (lane == 0) observed[1] = seen ? 1u : 0u;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_wait_timeout_probe(uint64_t limit_ns, int code, uint32_t *observed_dev, cudaStream_t stream) {
+    wait_timeout_probe_kernel<<<1, 64, 0, stream>>>(limit_ns, code, observed_dev);
+    return cudaGetLastError();
+}
 
 bool project_tc_applies(int32_t n_group, int32_t m) {
     // enough machines for the tensor core to pay, enough vectors to fill most of the 128 rows of the

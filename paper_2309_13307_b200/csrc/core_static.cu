@@ -5,8 +5,10 @@
 // application's memory pool owns all device memory, or inside a region where cudaMalloc's
 // implicit device synchronisation is not acceptable (a latency-critical loop, a library hook
 // that must not touch the allocator).  For them the partial sums live in the fixed array below,
-// which is part of the library image: every GPU that loads the library holds these 4 MiB until
-// the process exits, whether or not the entry point is ever called.
+// which is part of the library image: every GPU onto which this module has been loaded holds these
+// 4 MiB until the process exits.  With CUDA's default lazy module loading that happens at the first
+// cudaGetSymbolAddress below (first call of the entry point on that device), with eager loading when
+// the library is loaded.
 //
 // The array's name is a device symbol.  In host code it is only a handle, not a device
 // address, so the address the kernels receive is looked up once per device with
@@ -54,6 +56,17 @@ int scratch_for_current_device(float **out, int *device_out, int *last_cuda) {
     return CORE_OK;
 }
 
+// Is p device memory of `device`?  (Managed memory is accepted: it is reachable from every device.)
+bool on_device_memory(const void *p, int device) {
+    cudaPointerAttributes attr{};
+    if (cudaPointerGetAttributes(&attr, p) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    if (attr.type == cudaMemoryTypeManaged) return true;
+    return attr.type == cudaMemoryTypeDevice && attr.device == device;
+}
+
 }  // namespace
 
 extern "C" {
@@ -74,6 +87,8 @@ int core_project_static(uint64_t seed, uint32_t t, int64_t d, int32_t m, const v
         if (cuda_error_out) *cuda_error_out = last_cuda;
         return rc;
     }
+    // the scratch address belongs to the current device: so must the caller's buffers
+    if (!on_device_memory(G_dev, device) || !on_device_memory(P_dev, device)) return CORE_EINVAL;
     int sm_count = 0;
     cudaError_t e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, device);
     if (e != cudaSuccess) {
