@@ -144,3 +144,37 @@ def lipschitz_constant(A: torch.Tensor, iters: int = 100) -> float:
         lam = float(torch.linalg.norm(w))
         v = w / lam
     return lam
+
+
+def gossip_matrix(topology: str, n: int) -> np.ndarray:
+    """A network for the decentralised variant, given as its gossip matrix W (n x n float64, symmetric,
+    doubly stochastic, W[i][l] = 0 unless machines i and l are neighbours or i = l).
+
+    "ring":     machine i talks to i-1 and i+1 (mod n); weights 1/3 on each neighbour and on itself
+                (for n = 2 the two neighbours coincide: 1/2 and 1/2; n = 1: the 1 x 1 identity).
+    "torus":    machines on an a x b grid with wrap-around, a the largest divisor of n not above
+                sqrt(n); weight 1/5 on each of the four grid neighbours, the rest on itself
+                (coinciding neighbours add up).
+    "complete": every machine talks to every other: all weights 1/n (one round reaches the mean).
+    """
+    W = np.zeros((n, n), dtype=np.float64)
+    if topology == "complete":
+        W[:] = 1.0 / n
+        return W
+    if topology == "ring":
+        for i in range(n):
+            for l in ((i - 1) % n, (i + 1) % n):
+                W[i, l] += 1.0 / 3.0
+    elif topology == "torus":
+        a = max(k for k in range(1, int(np.sqrt(n)) + 1) if n % k == 0)
+        b = n // a
+        for i in range(n):
+            r, c = divmod(i, b)
+            for l in (((r - 1) % a) * b + c, ((r + 1) % a) * b + c, r * b + (c - 1) % b, r * b + (c + 1) % b):
+                W[i, l] += 1.0 / 5.0
+    else:
+        raise ValueError(topology)
+    for i in range(n):
+        W[i, i] = 0.0
+        W[i, i] = 1.0 - W[i].sum()
+    return W

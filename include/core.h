@@ -302,7 +302,7 @@ int core_debug_project_plan(int32_t n, int32_t m, int64_t d, int dtype, int32_t 
 /*
  * Instruction-rate probes (no counterpart in the paper: they support the roofline of the round kernels,
  * which are bound by instruction issue).  Kind k < core_debug_pipe_kinds() - 3 runs a loop whose body
- * is counts_out[0..6] = (32x32->64-bit multiplies, fp32 multiply-adds, packed fp32 multiply-adds,
+ * is counts_out[0..6] = (32x32-bit multiplies keeping the high word, fp32 multiply-adds, packed fp32 multiply-adds,
  * three-input logic ops, special-function calls, fp64 multiply-adds, 32-bit integer multiply-adds),
  * all on independent chains (core_debug_pipe_mix reports the counts, all zero for the last three
  * kinds).  The last three kinds run rounds 2..9 of Philox for four counters per body with the wide

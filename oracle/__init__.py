@@ -84,6 +84,18 @@ def lib() -> ctypes.CDLL:
             L.oracle_agd_step.restype = None
             L.oracle_gd_step_guarded.argtypes = [u64, u32, i32, vp, vp, i32, i32, i64, dbl, vp, vp, vp]
             L.oracle_gd_step_guarded.restype = ci
+            L.oracle_message_norm.argtypes = [vp, i32]
+            L.oracle_message_norm.restype = dbl
+            L.oracle_option1_step.argtypes = [dbl, i32, i64, dbl, dbl, dbl]
+            L.oracle_option1_step.restype = dbl
+            L.oracle_gd_step_option1.argtypes = [u64, u32, i32, vp, vp, i32, i32, i64, dbl, dbl, dbl, vp, vp, vp, vp, vp]
+            L.oracle_gd_step_option1.restype = ci
+            L.oracle_gossip_round.argtypes = [vp, vp, i32, i32, vp]
+            L.oracle_gossip_round.restype = None
+            L.oracle_gossip_average.argtypes = [vp, i32, i32, i32, vp, vp]
+            L.oracle_gossip_average.restype = None
+            L.oracle_decentralized_step.argtypes = [u64, u32, i32, vp, vp, i32, i32, i64, vp, i32, i32, ci, dbl, vp, vp]
+            L.oracle_decentralized_step.restype = dbl
             _lib = L
     return _lib
 
@@ -262,3 +274,63 @@ def gd_step_guarded(seed: int, t: int, m: int, A, b, h: float, x: np.ndarray, f_
     acc = lib().oracle_gd_step_guarded(seed, t, m, _ptr(A), _ptr(b), n, rows, d, float(h), _ptr(x), _ptr(f),
                                        _ptr(work))
     return x, float(f[0]), bool(acc)
+
+
+# ---- Algorithm 3, Option I -------------------------------------------------------
+
+def message_norm(pbar: np.ndarray) -> float:
+    """sqrt((1/m) sum_j pbar_j^2): the statistic p of Algorithm 3 in the reading taken here."""
+    pbar = np.ascontiguousarray(pbar, dtype=np.float64)
+    return lib().oracle_message_norm(_ptr(pbar), pbar.shape[0])
+
+
+def option1_step(p: float, m: int, d: int, r1: float, H: float, c: float = 1.0 / 1600.0) -> float:
+    return lib().oracle_option1_step(float(p), int(m), int(d), float(r1), float(H), float(c))
+
+
+def gd_step_option1(seed: int, t: int, m: int, A, b, r1: float, H: float, c: float, x: np.ndarray, f_x: float):
+    """One Algorithm-3 iteration with Option I: returns (x_kept, f(x_kept), accepted, p, h)."""
+    A, b, n, rows, d = _ls_arrays(A, b)
+    x = np.array(x, dtype=np.float64, copy=True)
+    f = np.array([f_x], dtype=np.float64)
+    p = np.zeros(1, dtype=np.float64)
+    h = np.zeros(1, dtype=np.float64)
+    work = np.zeros(n * d + n * m + m + 2 * d, dtype=np.float64)
+    acc = lib().oracle_gd_step_option1(seed, t, m, _ptr(A), _ptr(b), n, rows, d, float(r1), float(H), float(c),
+                                       _ptr(x), _ptr(f), _ptr(p), _ptr(h), _ptr(work))
+    return x, float(f[0]), bool(acc), float(p[0]), float(h[0])
+
+
+# ---- Algorithm 5: decentralised CORE-GD --------------------------------------------
+
+def gossip_round(W: np.ndarray, P: np.ndarray) -> np.ndarray:
+    W = np.ascontiguousarray(W, dtype=np.float64)
+    P = np.ascontiguousarray(P, dtype=np.float64)
+    n, m = P.shape
+    assert W.shape == (n, n)
+    out = np.zeros_like(P)
+    lib().oracle_gossip_round(_ptr(W), _ptr(P), n, m, _ptr(out))
+    return out
+
+
+def gossip_average(W: np.ndarray, P: np.ndarray, rounds: int) -> np.ndarray:
+    W = np.ascontiguousarray(W, dtype=np.float64)
+    P = np.array(P, dtype=np.float64, copy=True, order="C")
+    n, m = P.shape
+    assert W.shape == (n, n)
+    scratch = np.zeros_like(P)
+    lib().oracle_gossip_average(_ptr(W), int(rounds), n, m, _ptr(P), _ptr(scratch))
+    return P
+
+
+def decentralized_step(seed: int, t: int, m: int, A, b, W: np.ndarray, rounds: int, h: float, x: np.ndarray,
+                       reader: int = 0, as_printed: bool = False):
+    """One Algorithm-5 iteration; returns (x_new, spread of the machines' estimates around the reader's)."""
+    A, b, n, rows, d = _ls_arrays(A, b)
+    W = np.ascontiguousarray(W, dtype=np.float64)
+    assert W.shape == (n, n)
+    x = np.array(x, dtype=np.float64, copy=True)
+    work = np.zeros(n * d + 2 * n * m + d, dtype=np.float64)
+    spread = lib().oracle_decentralized_step(seed, t, m, _ptr(A), _ptr(b), n, rows, d, _ptr(W), int(rounds),
+                                             int(reader), 1 if as_printed else 0, float(h), _ptr(x), _ptr(work))
+    return x, float(spread)

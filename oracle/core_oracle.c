@@ -261,3 +261,94 @@ int oracle_gd_step_guarded(uint64_t seed, uint32_t t, int32_t m, const float *A,
     }
     return 0;
 }
+
+/* ---- Algorithm 3, Option I: the step chosen from the size of the messages ------ */
+
+double oracle_message_norm(const double *pbar, int32_t m) {
+    double sum_sq = 0.0;
+    for (int32_t j = 0; j < m; ++j) sum_sq += pbar[j] * pbar[j];
+    return sqrt(sum_sq / (double)m);
+}
+
+double oracle_option1_step(double p, int32_t m, int64_t d, double r1, double H, double c) {
+    double first = (double)m / (16.0 * r1);
+    /* c * H^(-1/2) * p^(-1/2) * d^(-3/4) * m^(3/4); p = 0 (no gradient) makes it infinite */
+    double second = c * pow(H, -0.5) * pow(p, -0.5) * pow((double)d, -0.75) * pow((double)m, 0.75);
+    return first < second ? first : second;
+}
+
+int oracle_gd_step_option1(uint64_t seed, uint32_t t, int32_t m, const float *A, const float *b, int32_t n,
+                           int32_t rows, int64_t d, double r1, double H, double c, double *x, double *f_x,
+                           double *p_out, double *h_out, double *work) {
+    double *G = work;                      /* n*d */
+    double *P = G + (size_t)n * (size_t)d; /* n*m */
+    double *pbar = P + (size_t)n * m;      /* m   */
+    double *gt = pbar + m;                 /* d   */
+    double *trial = gt + d;                /* d   */
+
+    /* the round: machine i sends p_ij, the central machine combines, everyone reconstructs */
+    oracle_ls_grad(A, b, n, rows, d, x, G);
+    oracle_project(seed, t, d, m, n, G, 2, d, P);
+    oracle_aggregate(P, n, m, pbar);
+    oracle_reconstruct_slice(seed, t, m, pbar, 0, d, gt);
+    /* the statistic p of the combined messages and the step it selects */
+    double p = oracle_message_norm(pbar, m);
+    double h = oracle_option1_step(p, m, d, r1, H, c);
+    if (p_out) *p_out = p;
+    if (h_out) *h_out = h;
+    /* trial point and comparison step; a tie keeps x */
+    for (int64_t k = 0; k < d; ++k) trial[k] = x[k] - h * gt[k];
+    double f_trial = oracle_ls_loss(A, b, n, rows, d, trial);
+    if (f_trial < *f_x) {
+        for (int64_t k = 0; k < d; ++k) x[k] = trial[k];
+        *f_x = f_trial;
+        return 1;
+    }
+    return 0;
+}
+
+/* ---- Algorithm 5: decentralised CORE-GD ----------------------------------------- */
+
+void oracle_gossip_round(const double *W, const double *P, int32_t n, int32_t m, double *P_next) {
+    for (int32_t i = 0; i < n; ++i)
+        for (int32_t j = 0; j < m; ++j) {
+            double s = 0.0;
+            for (int32_t l = 0; l < n; ++l) s += W[(size_t)i * n + l] * P[(size_t)l * m + j];
+            P_next[(size_t)i * m + j] = s;
+        }
+}
+
+void oracle_gossip_average(const double *W, int32_t rounds, int32_t n, int32_t m, double *P, double *scratch) {
+    for (int32_t r = 0; r < rounds; ++r) {
+        oracle_gossip_round(W, P, n, m, scratch);
+        memcpy(P, scratch, (size_t)n * m * sizeof(double));
+    }
+}
+
+double oracle_decentralized_step(uint64_t seed, uint32_t t, int32_t m, const float *A, const float *b, int32_t n,
+                                 int32_t rows, int64_t d, const double *W, int32_t rounds, int32_t reader,
+                                 int as_printed, double h, double *x, double *work) {
+    double *G = work;                      /* n*d */
+    double *P = G + (size_t)n * (size_t)d; /* n*m */
+    double *scratch = P + (size_t)n * m;   /* n*m */
+    double *gt = scratch + (size_t)n * m;  /* d   */
+
+    /* machine i computes its projections locally */
+    oracle_ls_grad(A, b, n, rows, d, x, G);
+    oracle_project(seed, t, d, m, n, G, 2, d, P);
+    /* the m-dimensional averaging problem, solved approximately by gossip: row i becomes machine i's
+     * estimate of p = (1/n) sum_i p_i */
+    oracle_gossip_average(W, rounds, n, m, P, scratch);
+    const double *p = P + (size_t)reader * m;
+    double spread = 0.0;
+    for (int32_t i = 0; i < n; ++i)
+        for (int32_t j = 0; j < m; ++j) {
+            double dev = fabs(P[(size_t)i * m + j] - p[j]);
+            if (dev > spread) spread = dev;
+        }
+    /* reconstruction from the consensus value, prefactor 1/m (mean reading) or n/m (as printed) */
+    oracle_reconstruct_slice(seed, t, m, p, 0, d, gt);
+    double prefactor = as_printed ? (double)n : 1.0;
+    for (int64_t k = 0; k < d; ++k) x[k] -= h * prefactor * gt[k];
+    return spread;
+}

@@ -26,7 +26,9 @@
  * restatement, hand-evaluated rounds and the generator's published
  * known-answer vectors; the round against hand-expanded sums at d=8, m=3,
  * unit-vector probes, <gbar, gtilde> = (1/m) sum pbar_j^2, linearity, and the
- * estimator's first and second moments (Lemma 3.1, proof of Lemma 3.2).
+ * estimator's first and second moments (Lemma 3.1, proof of Lemma 3.2); the message-norm statistic by
+ * the law of the messages, Option I's step by its closed form, gossip by the spectrum of W (limit = the
+ * centralised mean, contraction at the second eigenvalue) and a hand-worked three-machine example.
  */
 #ifndef CORE_ORACLE_H
 #define CORE_ORACLE_H
@@ -133,6 +135,57 @@ void oracle_agd_step(uint64_t seed, uint32_t t, int32_t m, const float *A, const
  */
 int oracle_gd_step_guarded(uint64_t seed, uint32_t t, int32_t m, const float *A, const float *b, int32_t n,
                            int32_t rows, int64_t d, double h, double *x, double *f_x, double *work);
+
+/*
+ * Algorithm 3 with Option I: the step is chosen from a statistic p of the combined messages.  The
+ * algorithm prints p = (1/m) sum_{i<=m} (sum_{j<=n} p_ij): its index ranges are swapped, and a plain mean
+ * of zero-mean Gaussians cannot bound the gradient norm as the proof of the theorem needs.  Reading
+ * taken: the root mean square of the combined messages,
+ *     p = sqrt((1/m) sum_j pbar_j^2),   pbar_j = (1/n) sum_i p_ij,
+ * whose square has expectation ||mean gradient||^2 (the messages of a vector a are N(0, ||a||^2 I_m),
+ * lemma on the law of the messages in the privacy appendix).
+ */
+double oracle_message_norm(const double *pbar, int32_t m);
+
+/*
+ * Option I's step: h = min{ m / (16 r1), c H^(-1/2) p^(-1/2) d^(-3/4) m^(3/4) } with r1 the bound on the
+ * trace of the Hessian, H the Lipschitz constant of the Hessian and c the printed constant (1/1600).
+ */
+double oracle_option1_step(double p, int32_t m, int64_t d, double r1, double H, double c);
+
+/*
+ * One iteration of Algorithm 3 with Option I on the least-squares objective, in the algorithm's order:
+ * round t (project, combine, reconstruct), p, h, trial point x - h * gtilde, comparison step (a tie keeps
+ * x).  *f_x: f(x) on entry, f of the kept point on return; *p_out, *h_out (may be NULL) receive the
+ * statistic and the step.  Returns 1 if the trial point was taken.  work: n*d + n*m + m + 2*d doubles.
+ */
+int oracle_gd_step_option1(uint64_t seed, uint32_t t, int32_t m, const float *A, const float *b, int32_t n,
+                           int32_t rows, int64_t d, double r1, double H, double c, double *x, double *f_x,
+                           double *p_out, double *h_out, double *work);
+
+/*
+ * Decentralised CORE-GD (appendix "Decentralized CORE Based Algorithms", Algorithm 5).  The machines
+ * hold their messages p_i (rows of P, n x m) and obtain p = (1/n) sum_i p_i, the minimiser of the
+ * m-dimensional problem (1/n) sum_i 1/2 ||x - p_i||^2, by exchanging with neighbours only.  Here that
+ * solver is plain gossip averaging with a gossip matrix W (n x n, row-major, symmetric, doubly
+ * stochastic, zero between machines that are not neighbours):
+ *     one round:  P_next[i] = sum_l W[i][l] P[l]   (l ascending).
+ * oracle_gossip_average runs `rounds` of them in place (scratch: n*m doubles).
+ */
+void oracle_gossip_round(const double *W, const double *P, int32_t n, int32_t m, double *P_next);
+void oracle_gossip_average(const double *W, int32_t rounds, int32_t n, int32_t m, double *P, double *scratch);
+
+/*
+ * One iteration of Algorithm 5 on the least-squares objective with round index t: local projections,
+ * `rounds` gossip rounds, reconstruction from machine `reader`'s estimate of p, x <- x - h * estimate.
+ * as_printed = 0 reconstructs with prefactor 1/m (the mean convention of the Section-4 estimator, as
+ * everywhere in this oracle); as_printed != 0 uses the printed n/m.  Returns the largest absolute
+ * difference between any machine's estimate and the reader's (how far from consensus the gossip
+ * stopped).  work: n*d + 2*n*m + d doubles.
+ */
+double oracle_decentralized_step(uint64_t seed, uint32_t t, int32_t m, const float *A, const float *b, int32_t n,
+                                 int32_t rows, int64_t d, const double *W, int32_t rounds, int32_t reader,
+                                 int as_printed, double h, double *x, double *work);
 
 #ifdef __cplusplus
 }

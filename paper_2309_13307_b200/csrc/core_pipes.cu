@@ -5,7 +5,7 @@
 // warp runs a loop whose body is a fixed mix of independent dependent-chains (wide integer multiplies,
 // fp32 and packed fp32 multiply-adds, three-input logic, special-function calls, fp64 multiply-adds,
 // 32-bit integer multiply-adds), and reports the SM cycles it took; with W warps resident per scheduler
-// the scheduler's cost of one loop body is cycles / (iterations * W).  Cycle counts do not depend on the
+// the scheduler's cost of one loop body is (span of the SM's warps) / (iterations * W).  Cycle counts do not depend on the
 // clock frequency.  Two further probes run the Philox rounds of the generator alone, with the 32x32->64
 // multiply done by the integer multiplier or by the fp64 unit (see philox_probe_kernel).
 #include "core.h"
@@ -24,7 +24,7 @@ struct Mix {
 
 // Loop bodies on offer: index = `kind` of core_debug_pipe_cycles.
 constexpr Mix kMixes[] = {
-    {16, 0, 0, 0, 0, 0, 0},    //  0  wide multiply alone
+    {16, 0, 0, 0, 0, 0, 0},    //  0  integer multiply, high word (the multiplier of mul.wide.u32) alone
     {0, 64, 0, 0, 0, 0, 0},    //  1  fp32 multiply-add
     {0, 0, 32, 0, 0, 0, 0},    //  2  packed fp32 multiply-add (two lanes per instruction)
     {0, 0, 0, 64, 0, 0, 0},    //  3  three-input logic
@@ -49,9 +49,11 @@ constexpr Mix kMixes[] = {
 constexpr int kMixCount = sizeof(kMixes) / sizeof(kMixes[0]);
 constexpr int kPhiloxKinds = 3;   // kinds kMixCount .. kMixCount+2: the Philox probes
 
-__device__ __forceinline__ unsigned long long mad_wide(uint32_t a, uint32_t b, unsigned long long c) {
-    unsigned long long d;
-    asm volatile("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
+// High word of a 32x32-bit product plus an addend: one instruction on the multiplier that also executes
+// mul.wide.u32 (the full product would need a second instruction to fold its halves into the chain).
+__device__ __forceinline__ uint32_t mad_hi(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm volatile("mad.hi.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
     return d;
 }
 __device__ __forceinline__ float ffma_v(float a, float b, float c) {
@@ -85,6 +87,17 @@ __device__ __forceinline__ uint32_t imad_v(uint32_t a, uint32_t b, uint32_t c) {
     return d;
 }
 
+// A warp's start and end on its SM's cycle counter, with the SM's id: the schedulers do not advance their
+// warps evenly, so the cost of a loop is taken from the span between the first start and the last end on
+// an SM, not from any one warp.
+__device__ __forceinline__ void record_stamps(long long *stamps, uint32_t warp, long long t0, long long t1) {
+    uint32_t smid;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    stamps[3 * warp] = (long long)smid;
+    stamps[3 * warp + 1] = t0;
+    stamps[3 * warp + 2] = t1;
+}
+
 template <int N>
 struct Chains {
     static constexpr int value = N == 0 ? 1 : (N < 8 ? N : 8);   // independent chains per class
@@ -93,20 +106,20 @@ struct Chains {
 // One warp's loop: `iters` bodies of the mix, every class on its own independent chains.
 template <int KIND>
 __global__ void __launch_bounds__(256)
-mix_probe_kernel(int iters, uint32_t seed, long long *cycles, uint32_t *sink) {
+mix_probe_kernel(int iters, uint32_t seed, long long *stamps, uint32_t *sink) {
     constexpr Mix M = kMixes[KIND];
     constexpr int CW = Chains<M.wide>::value, CF = Chains<M.ffma>::value, CP = Chains<M.ffma2>::value,
                   CL = Chains<M.lop3>::value, CM = Chains<M.mufu>::value, CD = Chains<M.dfma>::value,
                   CI = Chains<M.imad>::value;
     const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x;
-    unsigned long long w[CW];
+    uint32_t w[CW];
     float f[CF];
     unsigned long long p[CP];
     uint32_t l[CL];
     float s[CM];
     double d[CD];
     uint32_t im[CI];
-    for (int c = 0; c < CW; ++c) w[c] = (unsigned long long)(tid * 2654435761u + seed + c) * 0x9E3779B97F4A7C15ull;
+    for (int c = 0; c < CW; ++c) w[c] = (tid * 2654435761u + seed + c) | 0x80000000u;
     for (int c = 0; c < CF; ++c) f[c] = 1.0f + 1e-3f * (float)((tid + c) & 255);
     for (int c = 0; c < CP; ++c) p[c] = ((unsigned long long)__float_as_uint(1.0f + 1e-3f * c) << 32) | __float_as_uint(0.5f + 1e-3f * (tid & 63));
     for (int c = 0; c < CL; ++c) l[c] = tid * 747796405u + seed * (c + 1);
@@ -133,7 +146,7 @@ mix_probe_kernel(int iters, uint32_t seed, long long *cycles, uint32_t *sink) {
         for (int st = 0; st < STEPS; ++st) {
             if ((st + 1) * M.wide / STEPS > st * M.wide / STEPS) {
                 const int c = (st * M.wide / STEPS) % CW;
-                w[c] = mad_wide((uint32_t)w[c], mult, w[c]);
+                w[c] = mad_hi(w[c], mult, 0x9E3779B9u);
             }
             if ((st + 1) * M.dfma / STEPS > st * M.dfma / STEPS) {
                 const int c = (st * M.dfma / STEPS) % CD;
@@ -163,7 +176,7 @@ mix_probe_kernel(int iters, uint32_t seed, long long *cycles, uint32_t *sink) {
     }
     const long long t1 = clock64();
     uint32_t acc = 0;
-    for (int c = 0; c < CW; ++c) acc ^= (uint32_t)w[c] ^ (uint32_t)(w[c] >> 32);
+    for (int c = 0; c < CW; ++c) acc ^= w[c];
     for (int c = 0; c < CF; ++c) acc ^= __float_as_uint(f[c]);
     for (int c = 0; c < CP; ++c) acc ^= (uint32_t)p[c] ^ (uint32_t)(p[c] >> 32);
     for (int c = 0; c < CL; ++c) acc ^= l[c];
@@ -171,7 +184,7 @@ mix_probe_kernel(int iters, uint32_t seed, long long *cycles, uint32_t *sink) {
     for (int c = 0; c < CD; ++c) acc ^= (uint32_t)__double2loint(d[c]) ^ (uint32_t)__double2hiint(d[c]);
     for (int c = 0; c < CI; ++c) acc ^= im[c];
     sink[tid] = acc;
-    if ((threadIdx.x & 31) == 0) cycles[tid >> 5] = t1 - t0;
+    if ((threadIdx.x & 31) == 0) record_stamps(stamps, tid >> 5, t0, t1);
 }
 
 // ---- Philox alone, with the 32x32 -> 64-bit multiply done three ways -----------------------------
@@ -219,7 +232,7 @@ struct ProbeArgs {
 // A warp's loop: four counters per iteration (four vectors, one coordinate block), rounds 2..9 of each.
 template <int MODE>
 __global__ void __launch_bounds__(256)
-philox_probe_kernel(const __grid_constant__ ProbeArgs a, long long *cycles, uint32_t *sink) {
+philox_probe_kernel(const __grid_constant__ ProbeArgs a, long long *stamps, uint32_t *sink) {
     const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x;
     const double ma_d = (double)kPhiloxMulA, mb_d = (double)kPhiloxMulB;
     const double two84 = 19342813113834066795298816.0, two52 = 4503599627370496.0;
@@ -244,17 +257,17 @@ philox_probe_kernel(const __grid_constant__ ProbeArgs a, long long *cycles, uint
     }
     const long long t1 = clock64();
     sink[tid] = acc0 ^ acc1 ^ acc2 ^ acc3;
-    if ((threadIdx.x & 31) == 0) cycles[tid >> 5] = t1 - t0;
+    if ((threadIdx.x & 31) == 0) record_stamps(stamps, tid >> 5, t0, t1);
 }
 
 template <int K = 0>
-cudaError_t launch_mix(int kind, int grid, int iters, uint32_t seed, long long *cycles, uint32_t *sink, cudaStream_t s) {
+cudaError_t launch_mix(int kind, int grid, int iters, uint32_t seed, long long *stamps, uint32_t *sink, cudaStream_t s) {
     if constexpr (K < kMixCount) {
         if (kind == K) {
-            mix_probe_kernel<K><<<grid, 256, 0, s>>>(iters, seed, cycles, sink);
+            mix_probe_kernel<K><<<grid, 256, 0, s>>>(iters, seed, stamps, sink);
             return cudaGetLastError();
         }
-        return launch_mix<K + 1>(kind, grid, iters, seed, cycles, sink, s);
+        return launch_mix<K + 1>(kind, grid, iters, seed, stamps, sink, s);
     } else {
         return cudaErrorInvalidValue;
     }
@@ -288,9 +301,9 @@ int core_debug_pipe_cycles(int kind, int warps_per_scheduler, int iters, uint32_
     const int ctas_per_sm = warps_per_scheduler * 4 / 8;
     const int grid = sm_count * ctas_per_sm;
     const size_t warps = (size_t)grid * 8, threads = (size_t)grid * 256;
-    long long *cycles = nullptr;
+    long long *cycles = nullptr;                                    // per warp: SM id, first and last cycle
     uint32_t *sink = nullptr;
-    if (cudaMalloc(reinterpret_cast<void **>(&cycles), warps * sizeof(long long)) != cudaSuccess) return CORE_ENOMEM;
+    if (cudaMalloc(reinterpret_cast<void **>(&cycles), 3 * warps * sizeof(long long)) != cudaSuccess) return CORE_ENOMEM;
     if (cudaMalloc(reinterpret_cast<void **>(&sink), threads * sizeof(uint32_t)) != cudaSuccess) {
         cudaFree(cycles);
         return CORE_ENOMEM;
@@ -309,9 +322,9 @@ int core_debug_pipe_cycles(int kind, int warps_per_scheduler, int iters, uint32_
         }
         if (e == cudaSuccess) e = cudaDeviceSynchronize();
     }
-    std::vector<long long> host(warps);
+    std::vector<long long> host(3 * warps);
     std::vector<uint32_t> words(threads);
-    if (e == cudaSuccess) e = cudaMemcpy(host.data(), cycles, warps * sizeof(long long), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) e = cudaMemcpy(host.data(), cycles, 3 * warps * sizeof(long long), cudaMemcpyDeviceToHost);
     if (e == cudaSuccess) e = cudaMemcpy(words.data(), sink, threads * sizeof(uint32_t), cudaMemcpyDeviceToHost);
     cudaFree(cycles);
     cudaFree(sink);
@@ -319,9 +332,23 @@ int core_debug_pipe_cycles(int kind, int warps_per_scheduler, int iters, uint32_
         cudaGetLastError();
         return CORE_ECUDA;
     }
+    // per SM: span from its first warp's start to its last warp's end, shared out over the bodies its
+    // schedulers issued (warps on that SM / 4 schedulers, times the iterations)
+    std::vector<long long> first(1024, 0), last(1024, 0), count(1024, 0);
+    for (size_t w = 0; w < warps; ++w) {
+        const long long sm = host[3 * w] & 1023;
+        if (!count[sm] || host[3 * w + 1] < first[sm]) first[sm] = host[3 * w + 1];
+        if (!count[sm] || host[3 * w + 2] > last[sm]) last[sm] = host[3 * w + 2];
+        count[sm] += 1;
+    }
     double sum = 0.0;
-    for (long long c : host) sum += (double)c;
-    *cycles_per_body_out = sum / (double)warps / (double)iters / (double)warps_per_scheduler;
+    int sms = 0;
+    for (int sm = 0; sm < 1024; ++sm)
+        if (count[sm]) {
+            sum += (double)(last[sm] - first[sm]) / ((double)count[sm] / 4.0 * (double)iters);
+            ++sms;
+        }
+    *cycles_per_body_out = sum / (double)sms;
     if (checksum_out) {
         uint32_t x = 0;
         for (uint32_t v : words) x = x * 0x01000193u ^ v;
