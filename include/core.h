@@ -240,12 +240,50 @@ int core_agd_step(core_ctx *ctx, core_ls *ls, float h, float beta, float *x_dev,
  * round (current t, then t <- t + 1); x <- argmin over {x, x~} of f, a tie keeping x.
  *   f_dev         one double: f(x) on entry, f of the kept point on return
  *   accepted_dev  one int32 (may be NULL): 1 if the trial point was taken
- * The comparison is made on the device; the call does not synchronise.  Option I's
- * adaptive step is not offered: the statistic it is built on is garbled in the
- * algorithm's text.
+ * The comparison is made on the device; the call does not synchronise.
  */
 int core_gd_step_guarded(core_ctx *ctx, core_ls *ls, float h, float *x_dev, double *f_dev,
                          int32_t *accepted_dev);
+
+/*
+ * The same iteration with Option I of Algorithm 3: the step is chosen from the size of the combined
+ * messages of this very round,
+ *     p = sqrt((1/m) sum_j pbar_j^2),   h = min{ m / (16 r1), c H^(-1/2) p^(-1/2) d^(-3/4) m^(3/4) },
+ * r1 a bound on the trace of the Hessian, H the Lipschitz constant of the Hessian, c the algorithm's
+ * constant (it prints 1/1600); all three > 0.  The algorithm's own line for p has its index ranges
+ * swapped and, read literally, is a mean of zero-mean numbers that cannot bound the gradient norm as
+ * the proof requires; the root mean square above is the reading taken (its square has expectation
+ * ||mean gradient||^2, by the law of the messages).  p and h are formed on the device (in double,
+ * stored as float) between aggregation and reconstruction; nothing synchronises.
+ *   f_dev, accepted_dev  as for core_gd_step_guarded
+ *   p_dev, h_dev         one float each (may be NULL): the statistic and the step of this iteration
+ */
+int core_gd_step_option1(core_ctx *ctx, core_ls *ls, double r1, double H, double c, float *x_dev, double *f_dev,
+                         int32_t *accepted_dev, float *p_dev, float *h_dev);
+
+/* ---- decentralised CORE-GD (appendix "Decentralized CORE Based Algorithms", Algorithm 5) ------- */
+
+/*
+ * One gossip round on the machines' messages: P_out[i*m + j] = sum_l W[i*n + l] P_in[l*m + j], l
+ * ascending, fp32.  W_dev: the n x n gossip matrix of the network, row-major (symmetric, doubly
+ * stochastic, zero between machines that are not neighbours); P_in_dev, P_out_dev: n x m, distinct.
+ * Repeated rounds solve the algorithm's m-dimensional averaging problem, whose solution is
+ * p = (1/n) sum_i p_i: every row tends to it at the rate of W's second largest eigenvalue modulus.
+ */
+int core_gossip_round(core_ctx *ctx, const float *W_dev, const float *P_in_dev, int32_t n, float *P_out_dev);
+
+/*
+ * One iteration of Algorithm 5 on the least-squares objective, all n machines simulated on this GPU:
+ * every machine projects its own gradient (current t), `rounds` gossip rounds with W_dev replace the
+ * central machine, machine `reader`'s estimate of p is reconstructed and x <- x - h * estimate (inside
+ * the reconstruction), then t <- t + 1.  The algorithm presumes the averaging problem solved to
+ * accuracy: spread_dev (one float, may be NULL) receives max_ij |estimate_i[j] - estimate_reader[j]|,
+ * which tells whether `rounds` was enough.  as_printed = 0: prefactor 1/m, the mean convention of the
+ * Section-4 estimator used everywhere in this library; as_printed != 0: the printed n/m (the same
+ * direction, n times as long).
+ */
+int core_decentralized_step(core_ctx *ctx, core_ls *ls, const float *W_dev, int32_t rounds, int32_t reader,
+                            int as_printed, float h, float *x_dev, float *spread_dev);
 
 /*
  * f(x) as a double, computed on the device in a fixed order (the objective of Algorithm 2's

@@ -44,6 +44,11 @@ _SIGNATURES = {
     "core_agd_step": ([_c.c_void_p, _c.c_void_p, _c.c_float, _c.c_float, _c.c_void_p, _c.c_void_p], _c.c_int),
     "core_gd_step_guarded": ([_c.c_void_p, _c.c_void_p, _c.c_float, _c.c_void_p, _c.c_void_p, _c.c_void_p],
                              _c.c_int),
+    "core_gd_step_option1": ([_c.c_void_p, _c.c_void_p, _c.c_double, _c.c_double, _c.c_double, _c.c_void_p, _c.c_void_p,
+                              _c.c_void_p, _c.c_void_p, _c.c_void_p], _c.c_int),
+    "core_gossip_round": ([_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_int32, _c.c_void_p], _c.c_int),
+    "core_decentralized_step": ([_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_int32, _c.c_int32, _c.c_int, _c.c_float,
+                                 _c.c_void_p, _c.c_void_p], _c.c_int),
     "core_ls_loss": ([_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p], _c.c_int),
     "core_ls_loss_host": ([_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p], _c.c_int),
     "core_reserve_workspace": ([_c.c_void_p, _c.c_int32, _c.c_int], _c.c_int),
@@ -308,6 +313,33 @@ class Core:
         self._check(lib().core_gd_step_guarded(self._h, ls._h, float(h), _dev(x_dev, torch.float32, self.d),
                                                _dev(f_dev, torch.float64, 1), acc), "core_gd_step_guarded")
         return x_dev, f_dev
+
+    def core_gd_step_option1(self, ls: "LeastSquares", r1: float, H: float, c: float, x_dev: torch.Tensor,
+                             f_dev: torch.Tensor, accepted_dev: torch.Tensor | None = None,
+                             p_dev: torch.Tensor | None = None, h_dev: torch.Tensor | None = None):
+        opt = lambda t, dt: ctypes.c_void_p(_dev(t, dt, 1)) if t is not None else None
+        self._check(lib().core_gd_step_option1(self._h, ls._h, float(r1), float(H), float(c),
+                                               _dev(x_dev, torch.float32, self.d), _dev(f_dev, torch.float64, 1),
+                                               opt(accepted_dev, torch.int32), opt(p_dev, torch.float32),
+                                               opt(h_dev, torch.float32)), "core_gd_step_option1")
+        return x_dev, f_dev
+
+    def core_gossip_round(self, W_dev: torch.Tensor, P_in_dev: torch.Tensor, P_out_dev: torch.Tensor | None = None):
+        n = P_in_dev.shape[0]
+        if P_out_dev is None:
+            P_out_dev = torch.empty_like(P_in_dev)
+        self._check(lib().core_gossip_round(self._h, _dev(W_dev, torch.float32, n * n),
+                                            _dev(P_in_dev, torch.float32, n * self.m), n,
+                                            _dev(P_out_dev, torch.float32, n * self.m)), "core_gossip_round")
+        return P_out_dev
+
+    def core_decentralized_step(self, ls: "LeastSquares", W_dev: torch.Tensor, rounds: int, h: float, x_dev: torch.Tensor,
+                                reader: int = 0, as_printed: bool = False, spread_dev: torch.Tensor | None = None):
+        sp = ctypes.c_void_p(_dev(spread_dev, torch.float32, 1)) if spread_dev is not None else None
+        self._check(lib().core_decentralized_step(self._h, ls._h, _dev(W_dev, torch.float32, ls.n * ls.n), int(rounds),
+                                                  int(reader), 1 if as_printed else 0, float(h),
+                                                  _dev(x_dev, torch.float32, self.d), sp), "core_decentralized_step")
+        return x_dev
 
     def core_ls_loss(self, ls: "LeastSquares", x_dev: torch.Tensor, loss_dev: torch.Tensor | None = None):
         if loss_dev is None:

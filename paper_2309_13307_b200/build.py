@@ -12,7 +12,7 @@ CSRC = os.path.join(PKG, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(PKG, "libcore_b200.so")
 SOURCES = ["core_api.cu", "core_project.cu", "core_project_mma.cu", "core_project_tc.cu", "core_reconstruct.cu", "core_ls.cu",
-           "core_static.cu", "core_pipes.cu"]
+           "core_static.cu", "core_pipes.cu", "core_variants.cu"]
 HEADERS = [os.path.join(CSRC, "core_rng.cuh"), os.path.join(CSRC, "core_internal.h"),
            os.path.join(INCLUDE, "core.h")]
 

@@ -44,6 +44,7 @@ struct core_ls {
     float *y;            // d: look-ahead point of the accelerated step / trial point of the guarded step
     double *f_trial;     // loss at the trial point
     int *accepted;       // 1 if the last guarded step took the trial point
+    float *step;         // step chosen on the device (Option I of Algorithm 3), then its statistic p
 };
 
 namespace {
@@ -268,10 +269,25 @@ int core_reconstruct(core_ctx *ctx, const float *pbar_dev, float *gtilde_dev) {
     return CORE_OK;
 }
 
+// A step chosen on the device from the combined messages, between aggregation and reconstruction
+// (Option I of Algorithm 3): h_dev receives the step, p_dev (may be null) the statistic.
+struct StepRule {
+    double r1, H, c;
+    float *p_dev;
+    float *h_dev;
+};
+
+static int apply_step_rule(core_ctx *ctx, const StepRule *rule, const float *pbar_dev) {
+    if (!rule) return CORE_OK;
+    CORE_CUDA(ctx, launch_option1_step(pbar_dev, ctx->m, ctx->d, rule->r1, rule->H, rule->c, rule->p_dev, rule->h_dev,
+                                       ctx->stream));
+    return CORE_OK;
+}
+
 // project -> aggregate -> reconstruct with the current t, then t <- t + 1.  With an epilogue the
 // reconstruction writes the optimiser update into `out` instead of the estimate.
 static int round_with_epilogue(core_ctx *ctx, const void *G_dev, int dtype, int32_t n, int64_t ldg, float *pbar_dev,
-                               float *out, const ReconstructEpilogue *epilogue) {
+                               float *out, const ReconstructEpilogue *epilogue, const StepRule *rule = nullptr) {
     const size_t pb = partial_bytes(ctx, n, ctx->d, dtype);
     const size_t Pb = round_up((size_t)n * ctx->m * sizeof(float), 256);
     if (int rc = ensure_workspace(ctx, pb + Pb)) return rc;
@@ -287,6 +303,7 @@ static int round_with_epilogue(core_ctx *ctx, const void *G_dev, int dtype, int3
         if (int rc = project_into(ctx, G_dev, dtype, n, ldg, ctx->d, 0, partial, P, false, ctx->stream)) return rc;
         CORE_CUDA(ctx, launch_aggregate(P, n, ctx->m, pbar_dev, ctx->stream));
     }
+    if (int rc = apply_step_rule(ctx, rule, pbar_dev)) return rc;
     CORE_CUDA(ctx, launch_reconstruct(ctx->keys, ctx->t, pbar_dev, ctx->m, 0, ctx->d, out, ctx->sm_count, ctx->stream,
                                       epilogue));
     ctx->t += 1;
@@ -462,6 +479,7 @@ int core_ls_create(core_ls **out, const float *A_dev, const float *b_dev, int32_
     ls->y = reinterpret_cast<float *>(base + res_b + part_b + G_b);
     ls->f_trial = reinterpret_cast<double *>(base + res_b + part_b + G_b + gt_b);
     ls->accepted = reinterpret_cast<int *>(base + res_b + part_b + G_b + gt_b + 16);
+    ls->step = reinterpret_cast<float *>(base + res_b + part_b + G_b + gt_b + 32);
     *out = ls;
     return CORE_OK;
 }
@@ -490,7 +508,8 @@ static int ls_gradients_into(core_ctx *ctx, core_ls *ls, const float *x_dev, flo
 // Gradients at x_eval, then the round with the given epilogue.  Where the single-pass gradient kernel
 // and the scalar projection both apply, the projection sums the per-row-range partial gradients while
 // it stages its tiles, so the machine gradients G are never written or read back.
-static int ls_round(core_ctx *ctx, core_ls *ls, const float *x_eval, float *out, const ReconstructEpilogue *epilogue) {
+static int ls_round(core_ctx *ctx, core_ls *ls, const float *x_eval, float *out, const ReconstructEpilogue *epilogue,
+                    const StepRule *rule = nullptr) {
     if (ls->n <= kMaxGroup && ls_fused_usable(ls->fused_plan, ls->A, x_eval, ls->part)) {
         const ProjectPlan plan = make_project_plan(ls->n, ctx->m, ctx->d, CORE_F32, ctx->sm_count);
         if (plan.mma == 0) {
@@ -501,6 +520,7 @@ static int ls_round(core_ctx *ctx, core_ls *ls, const float *x_eval, float *out,
             CORE_CUDA(ctx, launch_project(plan, ctx->keys, ctx->t, ls->part, CORE_F32, ls->n, ls->d, ctx->d, ctx->m, 0,
                                           partial, ctx->stream, ls->fused_plan.splits, 1.0f / (float)ls->rows));
             CORE_CUDA(ctx, launch_finish_aggregate(partial, plan.grid_x, ls->n, ctx->m, ctx->pbar, ctx->stream));
+            if (int rc = apply_step_rule(ctx, rule, ctx->pbar)) return rc;
             CORE_CUDA(ctx, launch_reconstruct(ctx->keys, ctx->t, ctx->pbar, ctx->m, 0, ctx->d, out, ctx->sm_count,
                                               ctx->stream, epilogue));
             ctx->t += 1;
@@ -508,7 +528,7 @@ static int ls_round(core_ctx *ctx, core_ls *ls, const float *x_eval, float *out,
         }
     }
     if (int rc = ls_gradients_into(ctx, ls, x_eval, ls->G)) return rc;
-    return round_with_epilogue(ctx, ls->G, CORE_F32, ls->n, ls->d, ctx->pbar, out, epilogue);
+    return round_with_epilogue(ctx, ls->G, CORE_F32, ls->n, ls->d, ctx->pbar, out, epilogue, rule);
 }
 
 int core_ls_gradients(core_ctx *ctx, core_ls *ls, const float *x_dev, float *G_out_dev) {
@@ -546,6 +566,69 @@ int core_gd_step_guarded(core_ctx *ctx, core_ls *ls, float h, float *x_dev, doub
     // decided on the device: no host synchronisation inside the step
     CORE_CUDA(ctx, launch_keep_better(ls->f_trial, ls->y, ls->d, f_dev, x_dev, ls->accepted, accepted_dev,
                                       ctx->stream));
+    return CORE_OK;
+}
+
+int core_gd_step_option1(core_ctx *ctx, core_ls *ls, double r1, double H, double c, float *x_dev, double *f_dev,
+                         int32_t *accepted_dev, float *p_dev, float *h_dev) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!ls || !x_dev || !f_dev || ls->d != ctx->d || ls->device != ctx->device || !(r1 > 0.0) || !(H > 0.0) ||
+        !(c > 0.0))
+        return CORE_EINVAL;
+    // the step is formed on the device between aggregation and reconstruction; the reconstruction reads it
+    // there and writes the trial point y = x - h * gtilde; x is left untouched until the comparison
+    const StepRule rule{r1, H, c, ls->step + 1, ls->step};
+    ReconstructEpilogue trial{x_dev, 0.f, nullptr, nullptr};
+    trial.step_dev = ls->step;
+    if (int rc = ls_round(ctx, ls, x_dev, ls->y, &trial, &rule)) return rc;
+    CORE_CUDA(ctx, launch_ls_residual(ls->A, ls->b, ls->y, ls->n, ls->rows, ls->d, ls->res, ctx->stream));
+    CORE_CUDA(ctx, launch_ls_loss(ls->res, ls->n, ls->rows, ls->f_trial, ctx->stream));
+    CORE_CUDA(ctx, launch_keep_better(ls->f_trial, ls->y, ls->d, f_dev, x_dev, ls->accepted, accepted_dev,
+                                      ctx->stream));
+    if (h_dev)
+        CORE_CUDA(ctx, cudaMemcpyAsync(h_dev, ls->step, sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream));
+    if (p_dev)
+        CORE_CUDA(ctx, cudaMemcpyAsync(p_dev, ls->step + 1, sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream));
+    return CORE_OK;
+}
+
+int core_gossip_round(core_ctx *ctx, const float *W_dev, const float *P_in_dev, int32_t n, float *P_out_dev) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!W_dev || !P_in_dev || !P_out_dev || P_in_dev == P_out_dev || n < 1) return CORE_EINVAL;
+    CORE_CUDA(ctx, launch_gossip_round(W_dev, P_in_dev, n, ctx->m, P_out_dev, ctx->stream));
+    return CORE_OK;
+}
+
+int core_decentralized_step(core_ctx *ctx, core_ls *ls, const float *W_dev, int32_t rounds, int32_t reader,
+                            int as_printed, float h, float *x_dev, float *spread_dev) {
+    if (int rc = check_ctx(ctx)) return rc;
+    if (!ls || !W_dev || !x_dev || ls->d != ctx->d || ls->device != ctx->device || rounds < 0 || reader < 0 ||
+        reader >= ls->n)
+        return CORE_EINVAL;
+    const int32_t n = ls->n;
+    const size_t pb = partial_bytes(ctx, n, ctx->d, CORE_F32);
+    const size_t Pb = round_up((size_t)n * ctx->m * sizeof(float), 256);
+    if (int rc = ensure_workspace(ctx, pb + 2 * Pb)) return rc;
+    float *partial = static_cast<float *>(ctx->ws);
+    float *P = reinterpret_cast<float *>(static_cast<char *>(ctx->ws) + pb);
+    float *P_next = reinterpret_cast<float *>(static_cast<char *>(ctx->ws) + pb + Pb);
+    // every machine projects its own gradient; nothing is combined centrally
+    if (int rc = ls_gradients_into(ctx, ls, x_dev, ls->G)) return rc;
+    if (int rc = project_into(ctx, ls->G, CORE_F32, n, ls->d, ctx->d, 0, partial, P, false, ctx->stream)) return rc;
+    // the m-dimensional averaging problem, by gossip with the neighbours: row i is machine i's estimate
+    for (int32_t r = 0; r < rounds; ++r) {
+        CORE_CUDA(ctx, launch_gossip_round(W_dev, P, n, ctx->m, P_next, ctx->stream));
+        float *swap = P;
+        P = P_next;
+        P_next = swap;
+    }
+    if (spread_dev) CORE_CUDA(ctx, launch_consensus_spread(P, n, ctx->m, reader, spread_dev, ctx->stream));
+    // reconstruction from the reader's estimate, update inside the kernel; the printed prefactor n/m is
+    // the mean convention's 1/m with an n times longer step
+    const ReconstructEpilogue update{x_dev, as_printed ? h * (float)n : h, nullptr, nullptr};
+    CORE_CUDA(ctx, launch_reconstruct(ctx->keys, ctx->t, P + (size_t)reader * ctx->m, ctx->m, 0, ctx->d, x_dev,
+                                      ctx->sm_count, ctx->stream, &update));
+    ctx->t += 1;
     return CORE_OK;
 }
 

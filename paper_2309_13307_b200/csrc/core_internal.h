@@ -76,11 +76,15 @@ cudaError_t launch_aggregate(const float *P, int32_t n, int32_t m, float *pbar, 
 //   out[k] = base[k] - step * gtilde[k]   (the optimiser update of Algorithms 2 and 4)
 // and, if shift_dst is set, shift_dst[k] = shift_src[k] first (x_prev <- x of Algorithm 4).
 // out may alias base and shift_src; all four arrays are indexed like out.
+// step_dev, when set, overrides step: the kernel reads the step from device memory (a step that an
+// earlier kernel of the same iteration chose, as in Option I of Algorithm 3), times step_scale.
 struct ReconstructEpilogue {
     const float *base;
     float step;
     const float *shift_src;
     float *shift_dst;
+    const float *step_dev = nullptr;
+    float step_scale = 1.0f;
 };
 cudaError_t launch_reconstruct(const RoundKeys &keys, uint32_t t, const float *pbar, int32_t m,
                                int64_t k_begin, int64_t k_end, float *out, int sm_count,
@@ -124,5 +128,15 @@ cudaError_t launch_keep_better(const double *f_trial, const float *trial, int64_
                                int *flag_scratch, int32_t *flag_out, cudaStream_t stream);
 // loss[0] = (1/n) sum_i 1/(2 rows) sum_r res_i[r]^2, summed in double in a fixed order
 cudaError_t launch_ls_loss(const float *res, int32_t n, int32_t rows, double *loss, cudaStream_t stream);
+
+// Option I of Algorithm 3: p_out[0] (may be null) = sqrt((1/m) sum_j pbar_j^2), h_out[0] =
+// min{ m / (16 r1), c H^-1/2 p^-1/2 d^-3/4 m^3/4 }, both formed on the device in double and stored as float.
+cudaError_t launch_option1_step(const float *pbar, int32_t m, int64_t d, double r1, double H, double c, float *p_out,
+                                float *h_out, cudaStream_t stream);
+// Algorithm 5's averaging by gossip: out[i*m + j] = sum_l W[i*n + l] in[l*m + j], l ascending (in != out).
+cudaError_t launch_gossip_round(const float *W, const float *in, int32_t n, int32_t m, float *out, cudaStream_t stream);
+// spread[0] = max_ij |P[i*m + j] - P[reader*m + j]|
+cudaError_t launch_consensus_spread(const float *P, int32_t n, int32_t m, int32_t reader, float *spread,
+                                    cudaStream_t stream);
 
 }  // namespace core

@@ -68,12 +68,13 @@ __device__ __forceinline__ void rec_step(const uint4 *entries, const QPart (&qp)
 __device__ __forceinline__ void emit_block(const ReconstructArgs &a, uint64_t q, uint64_t q_begin, float4 r) {
     const int64_t off = (int64_t)((q - q_begin) << 2);        // offset into out
     const int64_t k = (int64_t)(q << 2);
+    const float step = a.epi.base ? (a.epi.step_dev ? a.epi.step_scale * __ldg(a.epi.step_dev) : a.epi.step) : 0.f;
     if (a.vec_ok && k + 4 <= a.k_end) {
         float4 v = r;
         if (a.epi.base) {
             const float4 b = *reinterpret_cast<const float4 *>(a.epi.base + off);
-            v = make_float4(fmaf(-a.epi.step, r.x, b.x), fmaf(-a.epi.step, r.y, b.y),
-                            fmaf(-a.epi.step, r.z, b.z), fmaf(-a.epi.step, r.w, b.w));
+            v = make_float4(fmaf(-step, r.x, b.x), fmaf(-step, r.y, b.y),
+                            fmaf(-step, r.z, b.z), fmaf(-step, r.w, b.w));
             if (a.epi.shift_dst) {
                 const float4 s = *reinterpret_cast<const float4 *>(a.epi.shift_src + off);
                 *reinterpret_cast<float4 *>(a.epi.shift_dst + off) = s;
@@ -87,7 +88,7 @@ __device__ __forceinline__ void emit_block(const ReconstructArgs &a, uint64_t q,
             if (k + l >= a.k_end) continue;
             float v = vals[l];
             if (a.epi.base) {
-                v = fmaf(-a.epi.step, v, a.epi.base[off + l]);
+                v = fmaf(-step, v, a.epi.base[off + l]);
                 if (a.epi.shift_dst) a.epi.shift_dst[off + l] = a.epi.shift_src[off + l];
             }
             a.out[off + l] = v;
