@@ -56,3 +56,32 @@ def test_reference_arm_prints_on_rank_zero_only():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
                           "--steps", "1", "--warmup", "1"], env=env, capture_output=True, text=True, timeout=300)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_gpus_flag_starts_that_many_ranks_by_itself(tmp_path):
+    """`bench.py --gpus N` without a launcher starts N ranks with RANK / LOCAL_RANK / WORLD_SIZE set and a
+    common rendezvous; here the ranks are a small CPU script that meets over gloo, so the spawning logic runs
+    without a GPU.  And a rank count that differs from --gpus is refused."""
+    sys.path.insert(0, ROOT)
+    import bench
+    script = tmp_path / "rank.py"
+    script.write_text(
+        "import json, os, sys\n"
+        "import torch, torch.distributed as dist\n"
+        "dist.init_process_group('gloo')\n"
+        "t = torch.tensor([float(os.environ['RANK']) + 1.0])\n"
+        "dist.all_reduce(t)\n"
+        "json.dump({'rank': int(os.environ['RANK']), 'local': int(os.environ['LOCAL_RANK']),\n"
+        "           'world': dist.get_world_size(), 'sum': float(t.item()), 'argv': sys.argv[1:]},\n"
+        "          open(os.path.join(sys.argv[1], 'spawned%s.json' % os.environ['RANK']), 'w'))\n"
+        "print('line from rank', os.environ['RANK'])\n"
+        "dist.destroy_process_group()\n")
+    rc = bench.spawn_replicas([str(tmp_path), "--gpus", "2"], 2, entry=[sys.executable, str(script)])
+    assert rc == 0
+    for rank in range(2):
+        got = json.load(open(tmp_path / f"spawned{rank}.json"))
+        assert got == {"rank": rank, "local": rank, "world": 2, "sum": 3.0, "argv": [str(tmp_path), "--gpus", "2"]}
+    env = dict(os.environ, RANK="0", WORLD_SIZE="2", LOCAL_RANK="0")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--steps", "1"], env=env,
+                         capture_output=True, text=True, timeout=120)
+    assert out.returncode != 0 and "refusing" in out.stderr and out.stdout.strip() == ""
