@@ -120,10 +120,11 @@ int core_device_status(int32_t *status_out);
  *   P_dev   n*m floats, row-major.
  * fp32 multiply-add with two-level fp32 accumulation and a fixed reduction
  * order: results are bitwise reproducible for a given (n, m, d, dtype).
- * n > 16 is processed in groups of 16 machines.  A group of 9..16 machines
- * with m >= 64 forms its products on the tensor cores with every operand split
- * into a tf32 head and tail (same error bar, same reproducibility).  May grow
- * the workspace.
+ * Machines are processed in groups: up to 32 per pass where the tensor-memory
+ * kernel applies (9 or more machines, m >= 96), otherwise up to 16.  The
+ * tensor-core kernels form their products with every operand split into a tf32
+ * head and tail (same error bar, same reproducibility).  May grow the
+ * workspace.
  */
 int core_project(core_ctx *ctx, const void *G_dev, int dtype, int32_t n, int64_t ldg, float *P_dev);
 
@@ -301,6 +302,14 @@ int core_ls_gradients(core_ctx *ctx, core_ls *ls, const float *x_dev, float *G_o
 /* ---- failure paths, made on the host or bounded on the device (no counterpart in the paper) ---- */
 
 /*
+ * Which projection kernel later calls use: -1 the library's choice by shape (default), 0 the scalar
+ * kernel, 1 the warp-level tensor-core kernel where its shape limits allow, 2 the tensor-memory
+ * (tcgen05) kernel for every group of up to 32 machines.  Process-wide; for measuring where one kernel
+ * overtakes the other and for testing each on shapes the default would not give it.
+ */
+int core_debug_force_project_kernel(int kind);
+
+/*
  * The next `count` device allocations of this library fail as if the device were out of memory
  * (count = 0 switches this off).  Lets a test see CORE_ENOMEM from core_init, core_project,
  * core_round_host, core_ls_create ... without exhausting a GPU: a failing call launches nothing and
@@ -328,9 +337,9 @@ int core_debug_gaussians(core_ctx *ctx, uint32_t j, uint64_t q0, int64_t nq, flo
 int core_debug_box_muller(core_ctx *ctx, const uint32_t *words_dev, int64_t nb, float *z_dev);
 
 /*
- * Launch geometry the projection would use for n machines (one pass handles at most 16),
+ * Launch geometry the projection would use for the first pass over n machines (at most 32 per pass),
  * m vectors and d coordinates on a device with sm_count SMs.  Host-only: touches no device.
- * out[0..9] = machines per pass (rounded up to a power of two), vectors per thread,
+ * out[0..9] = machines per pass (rounded up to a power of two; 16 or 32 for the tensor-memory kernel), vectors per thread,
  * coordinate blocks per thread step, blocks per shared-memory tile, threads across
  * vectors, threads across blocks, CTAs across coordinates, CTAs across vectors,
  * tiles of d, dynamic shared memory bytes.

@@ -53,6 +53,7 @@ _SIGNATURES = {
     "core_ls_loss_host": ([_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p], _c.c_int),
     "core_reserve_workspace": ([_c.c_void_p, _c.c_int32, _c.c_int], _c.c_int),
     "core_debug_fail_allocations": ([_c.c_int], _c.c_int),
+    "core_debug_force_project_kernel": ([_c.c_int], _c.c_int),
     "core_debug_wait_timeout": ([_c.c_uint32, _c.c_int32, _c.POINTER(_c.c_uint32)], _c.c_int),
     "core_ls_gradients": ([_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p], _c.c_int),
     "core_debug_philox": ([_c.c_void_p, _c.c_uint32, _c.c_uint64, _c.c_int64, _c.c_void_p], _c.c_int),
@@ -156,6 +157,13 @@ def core_debug_pipe_cycles(kind: int, warps_per_scheduler: int = 4, iters: int =
     if rc != CORE_OK:
         raise CoreError(rc, "core_debug_pipe_cycles")
     return float(cyc.value), int(chk.value)
+
+
+def core_debug_force_project_kernel(kind: int) -> None:
+    """-1: by shape (default); 0: scalar; 1: warp-level tensor cores; 2: tensor-memory kernel."""
+    rc = lib().core_debug_force_project_kernel(int(kind))
+    if rc != CORE_OK:
+        raise CoreError(rc, "core_debug_force_project_kernel")
 
 
 def core_debug_fail_allocations(count: int) -> None:

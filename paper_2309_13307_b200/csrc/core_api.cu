@@ -108,8 +108,8 @@ size_t elem_size(int dtype) { return dtype == CORE_BF16 ? 2 : 4; }
 // Bytes of partial sums the projection of n machines needs (largest group of a pass).
 size_t partial_bytes(const core_ctx *ctx, int32_t n, int64_t d, int dtype) {
     size_t need = 0;
-    for (int32_t i0 = 0; i0 < n; i0 += kMaxGroup) {
-        const int32_t ng = n - i0 < kMaxGroup ? n - i0 : kMaxGroup;
+    for (int32_t i0 = 0, ng = 0; i0 < n; i0 += ng) {
+        ng = project_group(n - i0, ctx->m);
         const ProjectPlan plan = make_project_plan(ng, ctx->m, d, dtype, ctx->sm_count);
         const size_t b = (size_t)plan.grid_x * ng * ctx->m * sizeof(float);
         if (b > need) need = b;
@@ -121,8 +121,8 @@ size_t partial_bytes(const core_ctx *ctx, int32_t n, int64_t d, int dtype) {
 // sums go through `partial`; P (n*m) receives (or accumulates) the result.
 int project_into(core_ctx *ctx, const void *G, int dtype, int32_t n, int64_t ldg, int64_t d, uint64_t q_base,
                  float *partial, float *P, bool accumulate, cudaStream_t stream) {
-    for (int32_t i0 = 0; i0 < n; i0 += kMaxGroup) {
-        const int32_t ng = n - i0 < kMaxGroup ? n - i0 : kMaxGroup;
+    for (int32_t i0 = 0, ng = 0; i0 < n; i0 += ng) {
+        ng = project_group(n - i0, ctx->m);
         const ProjectPlan plan = make_project_plan(ng, ctx->m, d, dtype, ctx->sm_count);
         const char *rows = static_cast<const char *>(G) + (size_t)i0 * (size_t)ldg * elem_size(dtype);
         CORE_CUDA(ctx, launch_project(plan, ctx->keys, ctx->t, rows, dtype, ng, ldg, d, ctx->m, q_base, partial,
@@ -293,7 +293,7 @@ static int round_with_epilogue(core_ctx *ctx, const void *G_dev, int dtype, int3
     if (int rc = ensure_workspace(ctx, pb + Pb)) return rc;
     float *partial = static_cast<float *>(ctx->ws);
     float *P = reinterpret_cast<float *>(static_cast<char *>(ctx->ws) + pb);
-    if (n <= kMaxGroup) {
+    if (project_group(n, ctx->m) == n) {
         // one group of machines: the per-machine messages are not kept, so they are never written
         const ProjectPlan plan = make_project_plan(n, ctx->m, ctx->d, dtype, ctx->sm_count);
         CORE_CUDA(ctx, launch_project(plan, ctx->keys, ctx->t, G_dev, dtype, n, ldg, ctx->d, ctx->m, 0, partial,
@@ -651,6 +651,12 @@ int core_ls_loss_host(core_ctx *ctx, core_ls *ls, const float *x_dev, double *lo
 
 /* ---- run-time diagnostics ------------------------------------------------------ */
 
+int core_debug_force_project_kernel(int kind) {
+    if (kind < -1 || kind > 2) return CORE_EINVAL;
+    project_force_kernel(kind);
+    return CORE_OK;
+}
+
 int core_debug_fail_allocations(int count) {
     if (count < 0) return CORE_EINVAL;
     g_fail_allocations.store(count);
@@ -702,7 +708,7 @@ int core_debug_box_muller(core_ctx *ctx, const uint32_t *words_dev, int64_t nb, 
 
 int core_debug_project_plan(int32_t n, int32_t m, int64_t d, int dtype, int32_t sm_count, int64_t out[10]) {
     if (!out || n < 1 || m < 1 || d < 1 || sm_count < 1 || !valid_dtype(dtype)) return CORE_EINVAL;
-    const ProjectPlan p = make_project_plan(n < kMaxGroup ? n : kMaxGroup, m, d, dtype, sm_count);
+    const ProjectPlan p = make_project_plan(project_group(n, m), m, d, dtype, sm_count);
     const int64_t v[10] = {p.nb, p.jt, p.uq, p.tile_q, p.tj, p.tq, p.grid_x, p.grid_y, p.tiles, (int64_t)p.smem};
     for (int i = 0; i < 10; ++i) out[i] = v[i];
     return CORE_OK;

@@ -307,7 +307,7 @@ __global__ void aggregate_kernel(const float *__restrict__ P, int n, int m, floa
 // the same sums in the same order, so pbar is bitwise what the two kernels give.
 __global__ void finish_aggregate_kernel(const float *__restrict__ partial, int chunks, int n, int m,
                                         float *__restrict__ pbar) {
-    __shared__ float message[kMaxGroup][32];       // P[i][j] of this block's 32 vectors
+    __shared__ float message[kMaxGroupTc][32];     // P[i][j] of this block's 32 vectors
     const int j = blockIdx.x * 32 + threadIdx.x, i = threadIdx.y;
     const int64_t total = (int64_t)n * m;
     float p = 0.f;
@@ -329,13 +329,28 @@ int ilog2(int x) {
 
 }  // namespace
 
+namespace {
+int g_force_kernel = -1;
+}
+
+void project_force_kernel(int kind) { g_force_kernel = kind; }
+
+int32_t project_group(int32_t n_left, int32_t m) {
+    if (n_left > kMaxGroup && g_force_kernel != 0 && g_force_kernel != 1) {
+        const int32_t wide = n_left < kMaxGroupTc ? n_left : kMaxGroupTc;
+        if (g_force_kernel == 2 || project_tc_applies(wide, m)) return wide;
+    }
+    return n_left < kMaxGroup ? n_left : kMaxGroup;
+}
+
 ProjectPlan make_project_plan(int32_t n_group, int32_t m, int64_t d, int dtype, int sm_count) {
     ProjectPlan p{};
-    if (project_tc_applies(n_group, m)) {
-        fill_project_tc_plan(p, m, d, dtype, sm_count);
+    const bool tc = g_force_kernel == 2 ? n_group <= kMaxGroupTc : (g_force_kernel < 0 && project_tc_applies(n_group, m));
+    if (tc) {
+        fill_project_tc_plan(p, n_group, m, d, dtype, sm_count);
         return p;
     }
-    if (project_mma_applies(n_group, m)) {
+    if (g_force_kernel != 0 && n_group <= kMaxGroup && project_mma_applies(n_group, m)) {
         fill_project_mma_plan(p, m, d, dtype, sm_count);
         return p;
     }
@@ -428,7 +443,8 @@ cudaError_t launch_finish_project(const float *partial, int chunks, int32_t n, i
 
 cudaError_t launch_finish_aggregate(const float *partial, int chunks, int32_t n, int32_t m, float *pbar,
                                     cudaStream_t stream) {
-    finish_aggregate_kernel<<<(m + 31) / 32, dim3(32, kMaxGroup), 0, stream>>>(partial, chunks, n, m, pbar);
+    finish_aggregate_kernel<<<(m + 31) / 32, dim3(32, n > kMaxGroup ? kMaxGroupTc : kMaxGroup), 0, stream>>>(
+        partial, chunks, n, m, pbar);
     return cudaGetLastError();
 }
 

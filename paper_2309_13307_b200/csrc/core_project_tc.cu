@@ -28,17 +28,31 @@ namespace {
 constexpr int kTcWarps = 8;
 constexpr int kTcThreads = 32 * kTcWarps;
 constexpr int kTcVectors = 128;                 // M of the instruction = vectors per CTA
-constexpr int kTcN = 16;                        // N of the instruction = machines per pass
+constexpr int kTcMaxN = 32;                     // largest N of the instruction = machines per pass (16 or 32)
+constexpr int kTcMinMachines = 9;               // fewer machines: the scalar kernel is used
 constexpr int kTcStageBlocks = 8;               // coordinate blocks per stage: 32 coordinates = 128 B per row
-constexpr int kTcStages = 3;                    // ring of stage buffers
+constexpr int kTcMaxStages = 3;                 // ring of stage buffers (2 where three would not fit twice per SM)
 constexpr int kTcTileStages = 8;                // stages between two drains of the accumulators
 constexpr int kTcTileBlocks = kTcStageBlocks * kTcTileStages;       // 64 blocks = 256 coordinates
 constexpr uint32_t kTcPlaneA = kTcVectors * 128;                    // bytes of one plane of Xi per stage
-constexpr uint32_t kTcPlaneB = kTcN * 128;                          // bytes of one plane of G per stage
-constexpr uint32_t kTcStageBytes = 2 * kTcPlaneA + 2 * kTcPlaneB;
+// Geometry that depends on N (machines per pass: 16 or 32) and on the gradients' type.  bf16 gradients are
+// exact in tf32 and need one plane, fp32 gradients a head and a tail plane.
+template <int NT, bool BF16>
+struct TcShape {
+    static constexpr uint32_t kPlaneB = NT * 128;                      // bytes of one plane of G per stage
+    static constexpr int kPlanesB = BF16 ? 1 : 2;
+    static constexpr uint32_t kStageBytes = 2 * kTcPlaneA + kPlanesB * kPlaneB;
+    // two CTAs per SM leave each about 113 KB of shared memory
+    static constexpr int kStages = 3 * kStageBytes + 2048 <= 113 * 1024 ? 3 : 2;
+    static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 128 + 1024;   // + barriers + alignment slack
+    static constexpr uint32_t kTmemColumns = 4 * NT;                   // two buffers x (head, tail products) x N
+    static constexpr int kDrainWarps = NT > 16 ? 8 : 4;                // each takes 32 vectors x 16 machines
+    // Instruction descriptor: fp32 accumulator (1 at bit 4), tf32 A and B (2 at bits 7 and 10), both
+    // K-major, N >> 3 at bit 17, M >> 4 at bit 24.
+    static constexpr uint32_t kIdesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(NT >> 3) << 17) |
+                                       ((uint32_t)(kTcVectors >> 4) << 24);
+};
 constexpr uint32_t kTcBarrierBytes = 128;
-constexpr uint32_t kTcSmemBytes = kTcStages * kTcStageBytes + kTcBarrierBytes + 1024;   // + alignment slack
-constexpr uint32_t kTcTmemColumns = 64;         // two buffers x (head products, tail products) x 16 columns
 constexpr uint64_t kTcWaitLimitNs = 100ull * 1000 * 1000;   // a wait gives up after 100 ms of the global timer
 
 __device__ int g_tc_status;                     // 0, or the code of a wait that ran out
@@ -154,10 +168,6 @@ constexpr uint32_t kDescHi = (kSbo >> 4) | (1u << 14);
 __device__ __forceinline__ uint32_t plane_offset(int row, int c) {
     return (uint32_t)(row >> 3) * kSbo + (uint32_t)c * kLbo + (uint32_t)(row & 7) * 16u;
 }
-// Instruction descriptor: fp32 accumulator (1 at bit 4), tf32 A and B (2 at bits 7 and 10), both K-major,
-// N >> 3 at bit 17, M >> 4 at bit 24.
-constexpr uint32_t kIdesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kTcN >> 3) << 17) |
-                            ((uint32_t)(kTcVectors >> 4) << 24);
 
 __device__ __forceinline__ float tf32_head(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
 
@@ -169,16 +179,17 @@ __device__ __forceinline__ void store_split(uint32_t dst, const float4 &z) {
     st_shared_v4<U * 4 * kSbo + kTcPlaneA>(dst, z.x - hx, z.y - hy, z.z - hz, z.w - hw);
 }
 
-// Head and tail of four fp32 gradient values into the two G planes of a stage.
+// Head and tail of four fp32 gradient values into the two G planes (PLANE_B bytes apart) of a stage.
+template <uint32_t PLANE_B>
 __device__ __forceinline__ void store_split_b(uint32_t dst, float x, float y, float z, float w) {
     const float hx = tf32_head(x), hy = tf32_head(y), hz = tf32_head(z), hw = tf32_head(w);
     st_shared_v4(dst, hx, hy, hz, hw);
-    st_shared_v4<kTcPlaneB>(dst, x - hx, y - hy, z - hz, w - hw);
+    st_shared_v4<PLANE_B>(dst, x - hx, y - hy, z - hz, w - hw);
 }
 
 // One thread's piece of a ragged or unaligned stage (4 coordinates for fp32, 8 for bf16, from k0 on),
 // element by element, zero beyond d and beyond n.  Kept out of line: it is rare.
-template <typename GT>
+template <typename GT, uint32_t PLANE_B>
 __device__ __noinline__ void stage_piece_slowly(const GT *G, int64_t ldg, int64_t d, int n, int i, int64_t k0, uint32_t dst) {
     constexpr bool BF16 = sizeof(GT) == 2;
     for (int part = 0; part < (BF16 ? 2 : 1); ++part) {
@@ -198,7 +209,7 @@ __device__ __noinline__ void stage_piece_slowly(const GT *G, int64_t ldg, int64_
         if constexpr (BF16)
             st_shared_v4(dst + (uint32_t)part * kLbo, vals[0], vals[1], vals[2], vals[3]);
         else
-            store_split_b(dst, vals[0], vals[1], vals[2], vals[3]);
+            store_split_b<PLANE_B>(dst, vals[0], vals[1], vals[2], vals[3]);
     }
 }
 
@@ -215,10 +226,15 @@ __device__ __forceinline__ bool mbar_try_wait_patient(uint32_t bar, uint32_t par
     return ok != 0;
 }
 
-template <typename GT>
+template <typename GT, int NT>
 __global__ void __launch_bounds__(kTcThreads, 2)
 project_tc_kernel(const __grid_constant__ TcArgs a) {
     constexpr bool BF16 = sizeof(GT) == 2;
+    using Shape = TcShape<NT, BF16>;
+    constexpr int kTcStages = Shape::kStages;
+    constexpr uint32_t kTcStageBytes = Shape::kStageBytes, kTcPlaneB = Shape::kPlaneB;
+    constexpr uint32_t kTcTmemColumns = Shape::kTmemColumns, kIdesc = Shape::kIdesc;
+    constexpr int kDrainWarps = Shape::kDrainWarps;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;                    // stage buffers, 1024-byte aligned
@@ -240,7 +256,7 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_acc_full + 8 * b, kTcTileStages);          // one tcgen05.commit per stage of the tile
-            mbar_init(bar_acc_empty + 8 * b, 4);                     // one arrival per draining warp
+            mbar_init(bar_acc_empty + 8 * b, kDrainWarps);           // one arrival per draining warp
         }
         mbar_init(bar_done, kTcWarps);                               // one tcgen05.commit per warp at the end
         *abort_flag = 0;
@@ -288,20 +304,23 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
         return ok;
     };
 
-    float outer[kTcN];
+    // A draining warp owns 32 vectors (its quarter of the tensor-memory lanes) x 16 machines (columns
+    // col0 .. col0 + 15: with 32 machines the upper four warps take the second half).
+    float outer[16];
 #pragma unroll
-    for (int c = 0; c < kTcN; ++c) outer[c] = 0.f;
+    for (int c = 0; c < 16; ++c) outer[c] = 0.f;
+    const uint32_t col0 = (uint32_t)(warp >> 2) * 16u;
     const int jbase = blockIdx.y * kTcVectors + lane;                // this thread's vectors: jbase + 32 u
-    auto drain = [&](int64_t local_tile) {                           // warps 0..3: tensor memory -> running sums
+    auto drain = [&](int64_t local_tile) {                           // draining warps: tensor memory -> running sums
         const uint32_t b = (uint32_t)(local_tile & 1);
         if (!warp_wait(bar_acc_full + 8 * b, (uint32_t)((local_tile >> 1) & 1), 3)) return;
         tc_fence_after_sync();
         float head[16], tail[16];
-        const uint32_t lane_base = taddr + ((uint32_t)(warp * 32) << 16) + b * (2 * kTcN);
+        const uint32_t lane_base = taddr + ((uint32_t)((warp & 3) * 32) << 16) + b * (2 * NT) + col0;
         tmem_load16(lane_base, head);
-        tmem_load16(lane_base + kTcN, tail);
+        tmem_load16(lane_base + NT, tail);
 #pragma unroll
-        for (int c = 0; c < kTcN; ++c) outer[c] += head[c] + tail[c];
+        for (int c = 0; c < 16; ++c) outer[c] += head[c] + tail[c];
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_acc_empty + 8 * b);
@@ -310,7 +329,7 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
     // Gradient staging is shared out among the warps in turn: DUTY warps serve a stage, one 16-byte piece
     // per thread, fetched one stage ahead so that the load is in flight while the previous stage is
     // generated.
-    constexpr int DUTY = BF16 ? 2 : 4;                              // warps on duty per stage
+    constexpr int DUTY = NT * (BF16 ? 4 : 8) / 32;                  // warps on duty per stage (one 16-byte piece per thread)
     constexpr uint32_t ROTA = kTcWarps / DUTY;                        // stages until a warp's turn comes again
     const uint32_t duty_phase = (uint32_t)warp / DUTY;                // serves stages c with c % ROTA == duty_phase
     const uint32_t fetch_phase = (duty_phase + ROTA - 1) % ROTA;      // and fetches for them one stage earlier
@@ -338,11 +357,11 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
                 st_shared_v4<kLbo>(dst, __uint_as_float(h.z << 16), __uint_as_float(h.z & 0xFFFF0000u),
                                    __uint_as_float(h.w << 16), __uint_as_float(h.w & 0xFFFF0000u));
             } else {
-                store_split_b(dst, __uint_as_float(h.x), __uint_as_float(h.y), __uint_as_float(h.z), __uint_as_float(h.w));
+                store_split_b<kTcPlaneB>(dst, __uint_as_float(h.x), __uint_as_float(h.y), __uint_as_float(h.z), __uint_as_float(h.w));
             }
             return;
         }
-        stage_piece_slowly<GT>(G, a.ldg, a.d, a.n, duty_i, range_begin + (int64_t)c * 32 + (BF16 ? 8 : 4) * duty_c, dst);
+        stage_piece_slowly<GT, kTcPlaneB>(G, a.ldg, a.d, a.n, duty_i, range_begin + (int64_t)c * 32 + (BF16 ? 8 : 4) * duty_c, dst);
     };
 
     // Products of one finished stage, issued by one lane.  `st` is the stage's index in its tile of
@@ -359,7 +378,7 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
                 // products with the head of xi and the head of g in one accumulator, the small products
                 // (a tail times a head) in another: the tensor core's accumulation error scales with the
                 // running sum, and the small ones then cost nothing
-                const uint32_t d_head = taddr + b * (2 * kTcN), d_tail = d_head + kTcN;
+                const uint32_t d_head = taddr + b * (2 * NT), d_tail = d_head + NT;
                 const uint32_t a_hi = smem_desc_lo(base + slot * kTcStageBytes);          // other planes: + bytes >> 4
                 const uint32_t a_lo = a_hi + (kTcPlaneA >> 4), b_hi = a_hi + (2 * kTcPlaneA >> 4);
                 const uint32_t b_lo = b_hi + (kTcPlaneB >> 4);
@@ -409,7 +428,7 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
             {
                 const uint32_t turn = count % ROTA;
                 if (turn == duty_phase) deposit(count, sb);
-                else if (turn == fetch_phase && count + 1 < total_stages) fetch(count + 1);
+                if (turn == fetch_phase && count + 1 < total_stages) fetch(count + 1);   // the same turn when all warps are on duty
             }
             const QPart qp = philox_qpart(q_lo, a.t, a.keys);
             uint4 w[4];
@@ -434,18 +453,20 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
             if (++s == kTcStages) { s = 0; ph ^= 1u; }
         }
         // the tile before this one has long been multiplied: fold it in while this one is in flight
-        if (alive && warp < 4 && tile > tile_begin) drain(tile - tile_begin - 1);
+        if (alive && warp < kDrainWarps && tile > tile_begin) drain(tile - tile_begin - 1);
     }
     if (alive && count > 0 && (uint32_t)warp == ((count - 1) & (kTcWarps - 1)))
         issue(prev_s, prev_ph, prev_st, prev_stages, prev_local);
-    if (alive && warp < 4 && tile_end > tile_begin) drain(tile_end - tile_begin - 1);
+    if (alive && warp < kDrainWarps && tile_end > tile_begin) drain(tile_end - tile_begin - 1);
 
-    if (warp < 4) {
-        const int j = blockIdx.y * kTcVectors + warp * 32 + lane;
+    if (warp < kDrainWarps) {
+        const int j = blockIdx.y * kTcVectors + (warp & 3) * 32 + lane;
         if (j < a.m) {
 #pragma unroll
-            for (int i = 0; i < kTcN; ++i)
-                if (i < a.n) a.partial[((int64_t)blockIdx.x * a.n + i) * a.m + j] = outer[i];
+            for (int c = 0; c < 16; ++c) {
+                const int i = (int)col0 + c;
+                if (i < a.n) a.partial[((int64_t)blockIdx.x * a.n + i) * a.m + j] = outer[c];
+            }
         }
     }
 
@@ -504,15 +525,16 @@ cudaError_t launch_wait_timeout_probe(uint64_t limit_ns, int code, uint32_t *obs
 }
 
 bool project_tc_applies(int32_t n_group, int32_t m) {
-    // enough machines for the tensor core to pay, enough vectors to fill most of the 128 rows of the
-    // last CTA row
-    return n_group > 8 && m >= 96 && (m % kTcVectors == 0 || m % kTcVectors >= 64 || m >= 1024);
+    // enough machines for the tensor core to pay (with five or more the multiply-adds of the scalar kernel cost
+    // more issue slots than this kernel's staging and hand-over), enough vectors to fill most of the 128 rows
+    // of the last CTA row
+    return n_group >= kTcMinMachines && n_group <= kTcMaxN && m >= 96 &&
+           (m % kTcVectors == 0 || m % kTcVectors >= 64 || m >= 1024);
 }
 
-void fill_project_tc_plan(ProjectPlan &p, int32_t m, int64_t d, int dtype, int sm_count) {
-    (void)dtype;
+void fill_project_tc_plan(ProjectPlan &p, int32_t n_group, int32_t m, int64_t d, int dtype, int sm_count) {
     p.mma = 2;
-    p.nb = kTcN;
+    p.nb = n_group > 16 ? 32 : 16;     // N of the instruction
     p.jt = 4;
     p.uq = 1;
     p.tile_q = kTcTileBlocks;
@@ -520,7 +542,9 @@ void fill_project_tc_plan(ProjectPlan &p, int32_t m, int64_t d, int dtype, int s
     p.tq = kTcWarps;
     p.grid_y = (m + kTcVectors - 1) / kTcVectors;
     p.tiles = (d + 4 * (int64_t)kTcTileBlocks - 1) / (4 * (int64_t)kTcTileBlocks);
-    p.smem = kTcSmemBytes;
+    const bool bf16 = dtype == 1;
+    p.smem = p.nb == 32 ? (bf16 ? TcShape<32, true>::kSmemBytes : TcShape<32, false>::kSmemBytes)
+                        : (bf16 ? TcShape<16, true>::kSmemBytes : TcShape<16, false>::kSmemBytes);
     int64_t gx = (int64_t)sm_count * 2 / p.grid_y;
     if (gx < 1) gx = 1;
     if (gx > p.tiles) gx = p.tiles;
@@ -530,7 +554,7 @@ void fill_project_tc_plan(ProjectPlan &p, int32_t m, int64_t d, int dtype, int s
 cudaError_t launch_project_tc(const ProjectPlan &plan, const RoundKeys &keys, uint32_t t, const void *G, int dtype,
                               int32_t n, int64_t ldg, int64_t d, int32_t m, uint64_t q_base, float *partial,
                               cudaStream_t stream) {
-    if (q_base % kTcTileBlocks != 0 || n > kTcN) return cudaErrorInvalidValue;
+    if (q_base % kTcTileBlocks != 0 || n > plan.nb || (plan.nb != 16 && plan.nb != 32)) return cudaErrorInvalidValue;
     TcArgs a{};
     a.G = G;
     a.ldg = ldg;
@@ -551,8 +575,12 @@ cudaError_t launch_project_tc(const ProjectPlan &plan, const RoundKeys &keys, ui
         kernel<<<grid, kTcThreads, plan.smem, stream>>>(a);
         return cudaGetLastError();
     };
-    if (dtype == 1) return go(project_tc_kernel<__nv_bfloat16>);
-    return go(project_tc_kernel<float>);
+    if (plan.nb == 32) {
+        if (dtype == 1) return go(project_tc_kernel<__nv_bfloat16, 32>);
+        return go(project_tc_kernel<float, 32>);
+    }
+    if (dtype == 1) return go(project_tc_kernel<__nv_bfloat16, 16>);
+    return go(project_tc_kernel<float, 16>);
 }
 
 cudaError_t project_tc_take_status(int *status) {

@@ -83,7 +83,12 @@ def test_ragged_sizes(core_mod, d, m, n):
     (12, 1024, 5_003, "f32", "normal"),          # more CTA rows than coordinate tiles per column
     (16, 384, 40_001, "f32", "scaled_normal"),
     (10, 200, 300, "bf16", "normal"),            # a single ragged tile; last CTA row 72 of 128 vectors
-    (41, 128, 2_049, "f32", "normal"),           # three passes, the last one scalar
+    (41, 128, 2_049, "f32", "normal"),           # a tensor-memory pass of 32 machines, then one of 9
+    (32, 256, 30_011, "f32", "scaled_normal"),   # 32 machines in one pass (N = 32 of the instruction), fp32: two-stage ring
+    (32, 256, 30_011, "bf16", "student_t3"),     # the same with one gradient plane and a three-stage ring
+    (50, 130, 9_001, "f32", "normal"),           # 32 + 18 machines
+    (64, 1024, 5_003, "bf16", "normal"),         # 32 + 32
+    (17, 96, 70_001, "bf16", "scaled_normal"),   # 17 machines: N = 32 with 15 empty columns
 ])
 def test_medium_sizes(core_mod, n, m, d, dtype, dist):
     G = core_inputs.gradients(n, d, seed=11, dist=dist, dtype=dtype, device="cuda")
@@ -120,6 +125,7 @@ def test_device_status_word(core_mod):
     (2, 8, "f32"), (4, 40, "bf16"), (8, 64, "f32"),       # scalar projection
     (10, 70, "f32"), (12, 72, "bf16"),                    # warp-level tensor-core projection
     (16, 256, "bf16"), (9, 128, "f32"),                   # tcgen05 projection
+    (32, 128, "f32"), (27, 256, "bf16"),                  # tcgen05 projection, 32 machines per pass
 ])
 def test_unit_vectors_read_the_generator_back(core_mod, n, m, dtype):
     """Machine i holds the unit vector e_k(i): its message is p_ij = xi_j[k(i)], and every other term of
@@ -204,6 +210,24 @@ def test_host_round_many_slabs(core_mod, m):
     for k0, k1 in [(0, 64), (2_097_100, 2_097_200), (d - 50, d)]:
         want = oracle.reconstruct_slice(4, 0, pbar_h.numpy().astype(np.float64), k0, k1)
         assert rel_l2(gt_h.numpy()[k0:k1], want) <= REC_TOL
+
+
+@pytest.mark.parametrize("kind,n,m,dtype", [(2, 5, 128, "f32"), (2, 8, 256, "bf16"), (2, 3, 40, "f32"), (2, 20, 33, "bf16"),
+                                          (0, 16, 256, "bf16"), (0, 12, 128, "f32"), (1, 16, 256, "f32")])
+def test_each_projection_kernel_on_shapes_the_default_would_not_give_it(core_mod, kind, n, m, dtype):
+    """The tensor-memory kernel with few machines and few vectors, the scalar and the warp-level kernels on
+    shapes that normally go to the tensor-memory kernel: all must meet the same bars."""
+    from paper_2309_13307_b200 import binding
+    G = core_inputs.gradients(n, 50_021, seed=21, dtype=dtype, device="cuda")
+    binding.core_debug_force_project_kernel(kind)
+    try:
+        plan = binding.core_debug_project_plan(n, m, 50_021, binding.CORE_BF16 if dtype == "bf16" else binding.CORE_F32,
+                                               torch.cuda.get_device_properties(0).multi_processor_count)
+        assert (plan["tj"] == 32 and plan["tq"] == 8 and plan["tile_q"] == 64) == (kind == 2)   # the tcgen05 geometry
+        check_round(core_mod, G, m, seed=9, t=4)
+    finally:
+        binding.core_debug_force_project_kernel(-1)
+    assert core_mod.lib().core_debug_force_project_kernel(3) == -1
 
 
 # ---- full-size workloads, sampled ---------------------------------------------------
