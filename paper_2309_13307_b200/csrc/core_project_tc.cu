@@ -1,8 +1,9 @@
 // Projection with the multiply-adds on the 5th-generation tensor cores (tcgen05 + tensor memory).
 //
 // For many machines the projection P = G Xi^T is a dense contraction whose operand Xi is generated on
-// the fly.  A CTA (8 warps) owns 128 vectors and a range of coordinates.  Per stage (128 vectors x 32
-// coordinates) every thread generates four counters' worth of Gaussians, splits each value into a tf32
+// the fly.  A CTA (8 warps) owns 128 or 256 vectors (one or two groups of 128, the M of the instruction)
+// and a range of coordinates.  Per stage (its vectors x 32 coordinates) every thread generates four or
+// eight counters' worth of Gaussians (one coordinate block, 4 or 8 vectors), splits each value into a tf32
 // head and tail (z = hi + lo, both exact in fp32) and writes the two planes to shared memory in the
 // K-major core-matrix layout the tensor core reads; in turn the warps also stage the machines' gradients
 // for the same 32 coordinates (split the same way when they are fp32; bf16 is exact in tf32).  The
@@ -21,38 +22,46 @@
 
 #include <cuda_bf16.h>
 
+#include <utility>
+
 namespace core {
 
 namespace {
 
 constexpr int kTcWarps = 8;
 constexpr int kTcThreads = 32 * kTcWarps;
-constexpr int kTcVectors = 128;                 // M of the instruction = vectors per CTA
+constexpr int kTcVectors = 128;                 // M of the instruction = vectors per group (a CTA owns VG groups)
 constexpr int kTcMaxN = 32;                     // largest N of the instruction = machines per pass (16 or 32)
 constexpr int kTcMinMachines = 9;               // fewer machines: the scalar kernel is used
 constexpr int kTcStageBlocks = 8;               // coordinate blocks per stage: 32 coordinates = 128 B per row
-constexpr int kTcMaxStages = 3;                 // ring of stage buffers (2 where three would not fit twice per SM)
 constexpr int kTcTileStages = 8;                // stages between two drains of the accumulators
 constexpr int kTcTileBlocks = kTcStageBlocks * kTcTileStages;       // 64 blocks = 256 coordinates
-constexpr uint32_t kTcPlaneA = kTcVectors * 128;                    // bytes of one plane of Xi per stage
-// Geometry that depends on N (machines per pass: 16 or 32) and on the gradients' type.  bf16 gradients are
-// exact in tf32 and need one plane, fp32 gradients a head and a tail plane.
-template <int NT, bool BF16>
+// Geometry that depends on N (machines per pass: 16 or 32), on the gradients' type and on VG (groups of
+// 128 vectors per CTA).  bf16 gradients are exact in tf32 and need one plane, fp32 gradients a head and a
+// tail plane.  With one group two CTAs share an SM (about 113 KB of shared memory each); with two groups a
+// CTA has the SM to itself, every thread generates eight counters per stage instead of four, and the
+// per-stage work that does not depend on the number of vectors (hand-over, issue, staging of the
+// gradients) is spread over twice as many Gaussians.
+template <int NT, bool BF16, int VG>
 struct TcShape {
+    static constexpr uint32_t kPlaneA = VG * kTcVectors * 128;         // bytes of one plane of Xi per stage
     static constexpr uint32_t kPlaneB = NT * 128;                      // bytes of one plane of G per stage
     static constexpr int kPlanesB = BF16 ? 1 : 2;
-    static constexpr uint32_t kStageBytes = 2 * kTcPlaneA + kPlanesB * kPlaneB;
-    // two CTAs per SM leave each about 113 KB of shared memory
-    static constexpr int kStages = 3 * kStageBytes + 2048 <= 113 * 1024 ? 3 : 2;
+    static constexpr uint32_t kStageBytes = 2 * kPlaneA + kPlanesB * kPlaneB;
+    static constexpr uint32_t kBudget = (VG == 1 ? 113u : 226u) * 1024u;
+    static constexpr int kStages = 3 * kStageBytes + 2048 <= kBudget ? 3 : 2;
     static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 128 + 1024;   // + barriers + alignment slack
-    static constexpr uint32_t kTmemColumns = 4 * NT;                   // two buffers x (head, tail products) x N
-    static constexpr int kDrainWarps = NT > 16 ? 8 : 4;                // each takes 32 vectors x 16 machines
+    static constexpr uint32_t kTmemColumns = 4 * NT * VG;              // two buffers x groups x (head, tail products) x N
+    // A draining warp reads its quarter of the tensor-memory lanes (32 vectors of a group) x 16 columns
+    // (machines): VG * NT / 16 such pieces per quarter, shared out over one or two warps per quarter.
+    static constexpr int kPieces = VG * NT / 16;
+    static constexpr int kDrainWarps = kPieces > 1 ? 8 : 4;
+    static constexpr int kPiecesPerWarp = kPieces > 2 ? kPieces / 2 : 1;
     // Instruction descriptor: fp32 accumulator (1 at bit 4), tf32 A and B (2 at bits 7 and 10), both
     // K-major, N >> 3 at bit 17, M >> 4 at bit 24.
     static constexpr uint32_t kIdesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(NT >> 3) << 17) |
                                        ((uint32_t)(kTcVectors >> 4) << 24);
 };
-constexpr uint32_t kTcBarrierBytes = 128;
 constexpr uint64_t kTcWaitLimitNs = 100ull * 1000 * 1000;   // a wait gives up after 100 ms of the global timer
 
 __device__ int g_tc_status;                     // 0, or the code of a wait that ran out
@@ -108,6 +117,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_
             if (mbar_try_wait(bar, parity)) return true;
     } while (global_timer_ns() - t0 < limit_ns);
     return false;
+}
+// True in exactly one lane of a converged warp.  Unlike a test of the lane index this keeps the branch, and the
+// operands computed for the instructions under it, warp-uniform in the compiler's eyes.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t chosen;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(chosen));
+    return chosen != 0;
 }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
@@ -171,12 +191,17 @@ __device__ __forceinline__ uint32_t plane_offset(int row, int c) {
 
 __device__ __forceinline__ float tf32_head(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
 
-// Head and tail of the four Gaussians of vector (lane + 32 U) into the two planes of a stage.
-template <int U>
+// Head and tail of the four Gaussians of vector (lane + 32 U) into the two planes (PLANE_A bytes apart)
+// of a stage.
+template <int U, uint32_t PLANE_A>
 __device__ __forceinline__ void store_split(uint32_t dst, const float4 &z) {
     const float hx = tf32_head(z.x), hy = tf32_head(z.y), hz = tf32_head(z.z), hw = tf32_head(z.w);
     st_shared_v4<U * 4 * kSbo>(dst, hx, hy, hz, hw);
-    st_shared_v4<U * 4 * kSbo + kTcPlaneA>(dst, z.x - hx, z.y - hy, z.z - hz, z.w - hw);
+    st_shared_v4<U * 4 * kSbo + PLANE_A>(dst, z.x - hx, z.y - hy, z.z - hz, z.w - hw);
+}
+template <uint32_t PLANE_A, int... U>
+__device__ __forceinline__ void store_split_all(uint32_t dst, const float4 *z, std::integer_sequence<int, U...>) {
+    (store_split<U, PLANE_A>(dst, z[U]), ...);
 }
 
 // Head and tail of four fp32 gradient values into the two G planes (PLANE_B bytes apart) of a stage.
@@ -213,28 +238,16 @@ __device__ __noinline__ void stage_piece_slowly(const GT *G, int64_t ldg, int64_
     }
 }
 
-// The same probe as mbar_try_wait, allowed to sleep in hardware for up to about `ns` before it answers.
-__device__ __forceinline__ bool mbar_try_wait_patient(uint32_t bar, uint32_t parity, uint32_t ns) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity), "r"(ns)
-        : "memory");
-    return ok != 0;
-}
-
-template <typename GT, int NT>
-__global__ void __launch_bounds__(kTcThreads, 2)
+template <typename GT, int NT, int VG>
+__global__ void __launch_bounds__(kTcThreads, VG == 1 ? 2 : 1)
 project_tc_kernel(const __grid_constant__ TcArgs a) {
     constexpr bool BF16 = sizeof(GT) == 2;
-    using Shape = TcShape<NT, BF16>;
+    using Shape = TcShape<NT, BF16, VG>;
     constexpr int kTcStages = Shape::kStages;
-    constexpr uint32_t kTcStageBytes = Shape::kStageBytes, kTcPlaneB = Shape::kPlaneB;
+    constexpr uint32_t kTcStageBytes = Shape::kStageBytes, kTcPlaneA = Shape::kPlaneA, kTcPlaneB = Shape::kPlaneB;
     constexpr uint32_t kTcTmemColumns = Shape::kTmemColumns, kIdesc = Shape::kIdesc;
-    constexpr int kDrainWarps = Shape::kDrainWarps;
+    constexpr int kDrainWarps = Shape::kDrainWarps, kPiecesPerWarp = Shape::kPiecesPerWarp;
+    constexpr int kCalls = 4 * VG;                                   // counters per thread and stage
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;                    // stage buffers, 1024-byte aligned
@@ -246,7 +259,9 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
     volatile uint32_t *const tmem_slot = words;                      // written by tcgen05.alloc
     volatile uint32_t *const abort_flag = words + 1;
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31;
+    // the warp's index, broadcast from a lane so that the compiler knows it to be the same in all lanes
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
     const GT *G = static_cast<const GT *>(a.G);
 
     if (tid == 0) {
@@ -266,7 +281,7 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    const uint32_t taddr = *tmem_slot;
+    const uint32_t taddr = __shfl_sync(0xffffffffu, *tmem_slot, 0);
 
     const int64_t per = (a.tiles + gridDim.x - 1) / gridDim.x;
     const int64_t tile_begin = (int64_t)blockIdx.x * per;
@@ -292,35 +307,31 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
         if (!ok && lane == 0) give_up(code);
         return ok;
     };
-    // One lane waits, patiently (the hardware may park it between probes).
-    auto lane_wait = [&](uint32_t bar, uint32_t parity, int code) {
-        bool ok = mbar_try_wait(bar, parity);
-        if (!ok) {
-            const uint64_t t0 = global_timer_ns();
-            do ok = mbar_try_wait_patient(bar, parity, 2000u);
-            while (!ok && global_timer_ns() - t0 < kTcWaitLimitNs);
-        }
-        if (!ok) give_up(code);
-        return ok;
-    };
-
-    // A draining warp owns 32 vectors (its quarter of the tensor-memory lanes) x 16 machines (columns
-    // col0 .. col0 + 15: with 32 machines the upper four warps take the second half).
-    float outer[16];
+    // A draining warp owns pieces of 32 vectors (its quarter of the tensor-memory lanes, in one group) x
+    // 16 machines: piece index = group * (NT / 16) + half of the columns.  With one piece per quarter
+    // warps 0..3 drain; with two, warps 4..7 take the second; with four, each warp takes two.
+    float outer[kPiecesPerWarp][16];
 #pragma unroll
-    for (int c = 0; c < 16; ++c) outer[c] = 0.f;
-    const uint32_t col0 = (uint32_t)(warp >> 2) * 16u;
-    const int jbase = blockIdx.y * kTcVectors + lane;                // this thread's vectors: jbase + 32 u
+    for (int r = 0; r < kPiecesPerWarp; ++r)
+#pragma unroll
+        for (int c = 0; c < 16; ++c) outer[r][c] = 0.f;
+    const int piece0 = (warp >> 2) * kPiecesPerWarp;                 // first piece of this warp
+    const int jbase = blockIdx.y * (VG * kTcVectors) + lane;         // this thread's vectors: jbase + 32 u
     auto drain = [&](int64_t local_tile) {                           // draining warps: tensor memory -> running sums
         const uint32_t b = (uint32_t)(local_tile & 1);
         if (!warp_wait(bar_acc_full + 8 * b, (uint32_t)((local_tile >> 1) & 1), 3)) return;
         tc_fence_after_sync();
-        float head[16], tail[16];
-        const uint32_t lane_base = taddr + ((uint32_t)((warp & 3) * 32) << 16) + b * (2 * NT) + col0;
-        tmem_load16(lane_base, head);
-        tmem_load16(lane_base + NT, tail);
 #pragma unroll
-        for (int c = 0; c < 16; ++c) outer[c] += head[c] + tail[c];
+        for (int r = 0; r < kPiecesPerWarp; ++r) {
+            const int piece = piece0 + r, g = piece / (NT / 16), half = piece % (NT / 16);
+            float head[16], tail[16];
+            const uint32_t lane_base = taddr + ((uint32_t)((warp & 3) * 32) << 16) + (b * VG + (uint32_t)g) * (2 * NT) +
+                                       (uint32_t)half * 16u;
+            tmem_load16(lane_base, head);
+            tmem_load16(lane_base + NT, tail);
+#pragma unroll
+            for (int c = 0; c < 16; ++c) outer[r][c] += head[c] + tail[c];
+        }
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_acc_empty + 8 * b);
@@ -367,35 +378,40 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
     // Products of one finished stage, issued by one lane.  `st` is the stage's index in its tile of
     // `stages`, `local` the tile's index in this CTA, (slot, parity) its ring position.
     auto issue = [&](uint32_t slot, uint32_t parity, int st, int stages, int64_t local) {
-        if (lane == 0) {
-            const uint32_t b = (uint32_t)(local & 1);
-            bool ok = true;
-            // the accumulators are free once the tile two back has been drained
-            if (st == 0) ok = lane_wait(bar_acc_empty + 8 * b, (uint32_t)(((local >> 1) & 1) ^ 1), 4);
-            if (ok) ok = lane_wait(bar_full + 8 * slot, parity, 5);
-            if (ok) {
-                tc_fence_after_sync();
-                // products with the head of xi and the head of g in one accumulator, the small products
-                // (a tail times a head) in another: the tensor core's accumulation error scales with the
-                // running sum, and the small ones then cost nothing
-                const uint32_t d_head = taddr + b * (2 * NT), d_tail = d_head + NT;
-                const uint32_t a_hi = smem_desc_lo(base + slot * kTcStageBytes);          // other planes: + bytes >> 4
-                const uint32_t a_lo = a_hi + (kTcPlaneA >> 4), b_hi = a_hi + (2 * kTcPlaneA >> 4);
-                const uint32_t b_lo = b_hi + (kTcPlaneB >> 4);
+        const uint32_t b = (uint32_t)(local & 1);
+        bool ok = true;
+        // the accumulators are free once the tile two back has been drained
+        if (st == 0) ok = warp_wait(bar_acc_empty + 8 * b, (uint32_t)(((local >> 1) & 1) ^ 1), 4);
+        if (ok) ok = warp_wait(bar_full + 8 * slot, parity, 5);
+        if (ok) {
+            tc_fence_after_sync();
+            // Everything up to the instructions themselves is computed by the whole warp from values that are
+            // the same in all lanes (descriptors then stay in uniform registers); one elected lane issues.
+            // Products with the head of xi and the head of g go to one accumulator, the small products (a
+            // tail times a head) to another: the tensor core's accumulation error scales with the running
+            // sum, and the small ones then cost nothing.
+            const uint32_t a_hi0 = smem_desc_lo(base + slot * kTcStageBytes);             // other planes: + bytes >> 4
+            const uint32_t b_hi = a_hi0 + (2 * kTcPlaneA >> 4), b_lo = b_hi + (kTcPlaneB >> 4);
+            if (elect_one()) {
 #pragma unroll
-                for (int kk = 0; kk < kTcStageBlocks / 2; ++kk) {
-                    const uint32_t step = (uint32_t)kk * 2u * kLbo >> 4;
-                    const uint32_t more = (st | kk) != 0;
-                    tc_mma_tf32(d_head, a_hi + step, b_hi + step, kDescHi, kIdesc, more);
-                    tc_mma_tf32(d_tail, a_lo + step, b_hi + step, kDescHi, kIdesc, more);
-                    if constexpr (!BF16) tc_mma_tf32(d_tail, a_hi + step, b_lo + step, kDescHi, kIdesc, 1u);
+                for (int g = 0; g < VG; ++g) {
+                    const uint32_t d_head = taddr + (b * VG + (uint32_t)g) * (2 * NT), d_tail = d_head + NT;
+                    const uint32_t a_hi = a_hi0 + (uint32_t)g * (kTcVectors * 128u >> 4), a_lo = a_hi + (kTcPlaneA >> 4);
+#pragma unroll
+                    for (int kk = 0; kk < kTcStageBlocks / 2; ++kk) {
+                        const uint32_t step = (uint32_t)kk * 2u * kLbo >> 4;
+                        const uint32_t more = (st | kk) != 0;
+                        tc_mma_tf32(d_head, a_hi + step, b_hi + step, kDescHi, kIdesc, more);
+                        tc_mma_tf32(d_tail, a_lo + step, b_hi + step, kDescHi, kIdesc, more);
+                        if constexpr (!BF16) tc_mma_tf32(d_tail, a_hi + step, b_lo + step, kDescHi, kIdesc, 1u);
+                    }
                 }
                 tc_commit(bar_empty + 8 * slot);                      // the stage buffer may be refilled
                 tc_commit(bar_acc_full + 8 * b);                      // one of the tile's kTcTileStages arrivals
                 if (st + 1 == stages)                                 // a short last tile: make up the count
                     for (int r = stages; r < kTcTileStages; ++r) tc_commit(bar_acc_full + 8 * b);
-                tc_fence_before_sync();                               // issued before this warp's arrival below
             }
+            tc_fence_before_sync();                                   // issued before this warp's arrival below
         }
         __syncwarp();
     };
@@ -408,9 +424,9 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
     int prev_st = 0, prev_stages = 0;
     int64_t prev_local = 0;
     uint32_t q_hi = (uint32_t)((a.q_base + (uint64_t)tile_begin * kTcTileBlocks) >> 32);
-    JPart jp[4];
+    JPart jp[kCalls];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) jp[u] = philox_jpart((uint32_t)(jbase + 32 * u), q_hi, a.keys);
+    for (int u = 0; u < kCalls; ++u) jp[u] = philox_jpart((uint32_t)(jbase + 32 * u), q_hi, a.keys);
     if (duty_phase == 0) fetch(0);
     bool alive = true;
     for (int64_t tile = tile_begin; tile < tile_end && alive; ++tile) {
@@ -418,7 +434,7 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
         if ((uint32_t)(q_tile >> 32) != q_hi) {                      // once per 2^32 blocks
             q_hi = (uint32_t)(q_tile >> 32);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) jp[u] = philox_jpart((uint32_t)(jbase + 32 * u), q_hi, a.keys);
+            for (int u = 0; u < kCalls; ++u) jp[u] = philox_jpart((uint32_t)(jbase + 32 * u), q_hi, a.keys);
         }
         const int stages = stages_of(tile);
         uint32_t q_lo = (uint32_t)q_tile + (uint32_t)warp;
@@ -431,16 +447,12 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
                 if (turn == fetch_phase && count + 1 < total_stages) fetch(count + 1);   // the same turn when all warps are on duty
             }
             const QPart qp = philox_qpart(q_lo, a.t, a.keys);
-            uint4 w[4];
+            uint4 w[kCalls];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) w[u] = philox_combine(jp[u], qp, a.keys);
-            float4 z[4];
-            box_muller4xN<4>(w, z);
-            const uint32_t dst = sb + row_off;
-            store_split<0>(dst, z[0]);
-            store_split<1>(dst, z[1]);
-            store_split<2>(dst, z[2]);
-            store_split<3>(dst, z[3]);
+            for (int u = 0; u < kCalls; ++u) w[u] = philox_combine(jp[u], qp, a.keys);
+            float4 z[kCalls];
+            box_muller4xN<kCalls>(w, z);
+            store_split_all<kTcPlaneA>(sb + row_off, z, std::make_integer_sequence<int, kCalls>{});
             // The previous stage's products go out before this warp reports the current stage done, so
             // that no other warp can be issuing a later stage first.
             if (count > 0 && (uint32_t)warp == ((count - 1) & (kTcWarps - 1))) {
@@ -460,18 +472,22 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
     if (alive && warp < kDrainWarps && tile_end > tile_begin) drain(tile_end - tile_begin - 1);
 
     if (warp < kDrainWarps) {
-        const int j = blockIdx.y * kTcVectors + (warp & 3) * 32 + lane;
-        if (j < a.m) {
 #pragma unroll
-            for (int c = 0; c < 16; ++c) {
-                const int i = (int)col0 + c;
-                if (i < a.n) a.partial[((int64_t)blockIdx.x * a.n + i) * a.m + j] = outer[c];
+        for (int r = 0; r < kPiecesPerWarp; ++r) {
+            const int piece = piece0 + r, g = piece / (NT / 16), half = piece % (NT / 16);
+            const int j = blockIdx.y * (VG * kTcVectors) + g * kTcVectors + (warp & 3) * 32 + lane;
+            if (j < a.m) {
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    const int i = half * 16 + c;
+                    if (i < a.n) a.partial[((int64_t)blockIdx.x * a.n + i) * a.m + j] = outer[r][c];
+                }
             }
         }
     }
 
     // nothing of this CTA may still be running on the tensor core when its tensor memory goes back
-    if (lane == 0) tc_commit(bar_done);
+    if (elect_one()) tc_commit(bar_done);                            // the lane that issued this warp's products
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) {
@@ -532,20 +548,33 @@ bool project_tc_applies(int32_t n_group, int32_t m) {
            (m % kTcVectors == 0 || m % kTcVectors >= 64 || m >= 1024);
 }
 
+// Two groups of 128 vectors per CTA (one CTA per SM) when that leaves few rows of the last CTA row
+// empty; otherwise one group (two CTAs per SM).
+static int tc_vector_groups(int32_t m) {
+    const int32_t rest = m % (2 * kTcVectors);
+    return (m >= 2 * kTcVectors && (rest == 0 || rest > kTcVectors + kTcVectors / 2 || m >= 16 * kTcVectors)) ? 2 : 1;
+}
+
+template <int NT, int VG>
+static size_t tc_smem_bytes(bool bf16) {
+    return bf16 ? TcShape<NT, true, VG>::kSmemBytes : TcShape<NT, false, VG>::kSmemBytes;
+}
+
 void fill_project_tc_plan(ProjectPlan &p, int32_t n_group, int32_t m, int64_t d, int dtype, int sm_count) {
+    const int vg = tc_vector_groups(m);
     p.mma = 2;
     p.nb = n_group > 16 ? 32 : 16;     // N of the instruction
-    p.jt = 4;
+    p.jt = 4 * vg;                     // producer thread = (lane, warp): 4 or 8 vectors x 1 block per stage
     p.uq = 1;
     p.tile_q = kTcTileBlocks;
-    p.tj = 32;                         // producer thread = (lane, warp): 4 vectors x 1 block per stage
+    p.tj = 32;
     p.tq = kTcWarps;
-    p.grid_y = (m + kTcVectors - 1) / kTcVectors;
+    p.grid_y = (m + vg * kTcVectors - 1) / (vg * kTcVectors);
     p.tiles = (d + 4 * (int64_t)kTcTileBlocks - 1) / (4 * (int64_t)kTcTileBlocks);
     const bool bf16 = dtype == 1;
-    p.smem = p.nb == 32 ? (bf16 ? TcShape<32, true>::kSmemBytes : TcShape<32, false>::kSmemBytes)
-                        : (bf16 ? TcShape<16, true>::kSmemBytes : TcShape<16, false>::kSmemBytes);
-    int64_t gx = (int64_t)sm_count * 2 / p.grid_y;
+    if (vg == 2) p.smem = p.nb == 32 ? tc_smem_bytes<32, 2>(bf16) : tc_smem_bytes<16, 2>(bf16);
+    else p.smem = p.nb == 32 ? tc_smem_bytes<32, 1>(bf16) : tc_smem_bytes<16, 1>(bf16);
+    int64_t gx = (int64_t)sm_count * (vg == 2 ? 1 : 2) / p.grid_y;
     if (gx < 1) gx = 1;
     if (gx > p.tiles) gx = p.tiles;
     p.grid_x = (int)gx;
@@ -554,7 +583,8 @@ void fill_project_tc_plan(ProjectPlan &p, int32_t n_group, int32_t m, int64_t d,
 cudaError_t launch_project_tc(const ProjectPlan &plan, const RoundKeys &keys, uint32_t t, const void *G, int dtype,
                               int32_t n, int64_t ldg, int64_t d, int32_t m, uint64_t q_base, float *partial,
                               cudaStream_t stream) {
-    if (q_base % kTcTileBlocks != 0 || n > plan.nb || (plan.nb != 16 && plan.nb != 32)) return cudaErrorInvalidValue;
+    if (q_base % kTcTileBlocks != 0 || n > plan.nb || (plan.nb != 16 && plan.nb != 32) || (plan.jt != 4 && plan.jt != 8))
+        return cudaErrorInvalidValue;
     TcArgs a{};
     a.G = G;
     a.ldg = ldg;
@@ -575,12 +605,17 @@ cudaError_t launch_project_tc(const ProjectPlan &plan, const RoundKeys &keys, ui
         kernel<<<grid, kTcThreads, plan.smem, stream>>>(a);
         return cudaGetLastError();
     };
-    if (plan.nb == 32) {
-        if (dtype == 1) return go(project_tc_kernel<__nv_bfloat16, 32>);
-        return go(project_tc_kernel<float, 32>);
-    }
-    if (dtype == 1) return go(project_tc_kernel<__nv_bfloat16, 16>);
-    return go(project_tc_kernel<float, 16>);
+    auto pick = [&](auto nt, auto vg) {
+        constexpr int NT = decltype(nt)::value, VG = decltype(vg)::value;
+        if (dtype == 1) return go(project_tc_kernel<__nv_bfloat16, NT, VG>);
+        return go(project_tc_kernel<float, NT, VG>);
+    };
+    using I16 = std::integral_constant<int, 16>;
+    using I32 = std::integral_constant<int, 32>;
+    using I1 = std::integral_constant<int, 1>;
+    using I2 = std::integral_constant<int, 2>;
+    if (plan.jt == 8) return plan.nb == 32 ? pick(I32{}, I2{}) : pick(I16{}, I2{});
+    return plan.nb == 32 ? pick(I32{}, I1{}) : pick(I16{}, I1{});
 }
 
 cudaError_t project_tc_take_status(int *status) {

@@ -89,6 +89,8 @@ def test_ragged_sizes(core_mod, d, m, n):
     (50, 130, 9_001, "f32", "normal"),           # 32 + 18 machines
     (64, 1024, 5_003, "bf16", "normal"),         # 32 + 32
     (17, 96, 70_001, "bf16", "scaled_normal"),   # 17 machines: N = 32 with 15 empty columns
+    (16, 456, 30_001, "f32", "normal"),          # two groups of 128 vectors per CTA, second CTA row 200 of 256 full
+    (20, 456, 30_001, "bf16", "student_t3"),     # the same with N = 32
 ])
 def test_medium_sizes(core_mod, n, m, d, dtype, dist):
     G = core_inputs.gradients(n, d, seed=11, dist=dist, dtype=dtype, device="cuda")
