@@ -120,8 +120,9 @@ int core_device_status(int32_t *status_out);
  *   P_dev   n*m floats, row-major.
  * fp32 multiply-add with two-level fp32 accumulation and a fixed reduction
  * order: results are bitwise reproducible for a given (n, m, d, dtype).
- * Machines are processed in groups: up to 32 per pass where the tensor-memory
- * kernel applies (9 or more machines, m >= 96), otherwise up to 16.  The
+ * Machines are processed in groups: up to 64 per pass where the tensor-memory
+ * kernel applies (9 or more machines, m >= 96; more than 32 only when m lets a CTA
+ * hold 256 vectors, about m >= 256), otherwise up to 16.  The
  * tensor-core kernels form their products with every operand split into a tf32
  * head and tail (same error bar, same reproducibility).  May grow the
  * workspace.
@@ -304,7 +305,7 @@ int core_ls_gradients(core_ctx *ctx, core_ls *ls, const float *x_dev, float *G_o
 /*
  * Which projection kernel later calls use: -1 the library's choice by shape (default), 0 the scalar
  * kernel, 1 the warp-level tensor-core kernel where its shape limits allow, 2 the tensor-memory
- * (tcgen05) kernel for every group of up to 32 machines.  Process-wide; for measuring where one kernel
+ * (tcgen05) kernel for every group of machines it can take (up to 64).  Process-wide; for measuring where one kernel
  * overtakes the other and for testing each on shapes the default would not give it.
  */
 int core_debug_force_project_kernel(int kind);
@@ -337,9 +338,9 @@ int core_debug_gaussians(core_ctx *ctx, uint32_t j, uint64_t q0, int64_t nq, flo
 int core_debug_box_muller(core_ctx *ctx, const uint32_t *words_dev, int64_t nb, float *z_dev);
 
 /*
- * Launch geometry the projection would use for the first pass over n machines (at most 32 per pass),
+ * Launch geometry the projection would use for the first pass over n machines (at most 64 per pass),
  * m vectors and d coordinates on a device with sm_count SMs.  Host-only: touches no device.
- * out[0..9] = machines per pass (rounded up to a power of two; 16 or 32 for the tensor-memory kernel), vectors per thread,
+ * out[0..9] = machines per pass (rounded up to a power of two; 16, 32 or 64 for the tensor-memory kernel), vectors per thread,
  * coordinate blocks per thread step, blocks per shared-memory tile, threads across
  * vectors, threads across blocks, CTAs across coordinates, CTAs across vectors,
  * tiles of d, dynamic shared memory bytes.

@@ -11,13 +11,13 @@ namespace core {
 
 constexpr int kThreads = 256;        // threads per CTA in the round kernels
 constexpr int kMaxGroup = 16;        // machines handled by one pass of the scalar projection
-constexpr int kMaxGroupTc = 32;      // machines handled by one pass of the tensor-memory projection
+constexpr int kMaxGroupTc = 64;      // most machines one pass of the tensor-memory projection can take
 
-// Machines the next projection pass takes when n_left remain: 32 where the tensor-memory kernel applies
-// to more than 16, otherwise at most 16.
+// Machines the next projection pass takes when n_left remain: up to 64 (32 where a CTA holds one group of
+// 128 vectors only) where the tensor-memory kernel applies to more than 16, otherwise at most 16.
 int32_t project_group(int32_t n_left, int32_t m);
 // Test hook: -1 = choose by shape (default); 0 = always the scalar kernel; 1 = the warp-level tensor-core
-// kernel where its shape limits allow; 2 = the tensor-memory kernel for any group of up to 32 machines.
+// kernel where its shape limits allow; 2 = the tensor-memory kernel for any group of machines it can take.
 void project_force_kernel(int kind);
 
 // Launch geometry of one projection pass, fixed by (n, m, d, dtype) on the host.
@@ -44,11 +44,12 @@ cudaError_t launch_project_mma(const ProjectPlan &plan, const RoundKeys &keys, u
                                int dtype, int32_t n, int64_t ldg, int64_t d, int32_t m, uint64_t q_base,
                                float *partial, cudaStream_t stream);
 
-// tcgen05 variant (core_project_tc.cu): 128 vectors per CTA, up to 32 machines per pass (N = 16 or 32 of
-// the instruction), accumulators in tensor memory; same partial-sum layout.  q_base must be a multiple of 64 blocks.  Its waits are bounded: a wait that
+// tcgen05 variant (core_project_tc.cu): 128 or 256 vectors per CTA, up to project_tc_max_group(m) machines per
+// pass (N = 16, 32 or 64 of the instruction), accumulators in tensor memory; same partial-sum layout.  q_base must be a multiple of 64 blocks.  Its waits are bounded: a wait that
 // runs out raises a device status word, which project_tc_take_status returns and clears after
 // synchronising the device.
 bool project_tc_applies(int32_t n_group, int32_t m);
+int32_t project_tc_max_group(int32_t m);   // 64 with 256 vectors per CTA, otherwise 32
 void fill_project_tc_plan(ProjectPlan &plan, int32_t n_group, int32_t m, int64_t d, int dtype, int sm_count);
 cudaError_t launch_project_tc(const ProjectPlan &plan, const RoundKeys &keys, uint32_t t, const void *G,
                               int dtype, int32_t n, int64_t ldg, int64_t d, int32_t m, uint64_t q_base,

@@ -308,14 +308,16 @@ __global__ void aggregate_kernel(const float *__restrict__ P, int n, int m, floa
 __global__ void finish_aggregate_kernel(const float *__restrict__ partial, int chunks, int n, int m,
                                         float *__restrict__ pbar) {
     __shared__ float message[kMaxGroupTc][32];     // P[i][j] of this block's 32 vectors
-    const int j = blockIdx.x * 32 + threadIdx.x, i = threadIdx.y;
+    const int j = blockIdx.x * 32 + threadIdx.x;
     const int64_t total = (int64_t)n * m;
-    float p = 0.f;
-    if (j < m && i < n)
-        for (int c = 0; c < chunks; ++c) p += partial[(int64_t)c * total + (int64_t)i * m + j];
-    message[i][threadIdx.x] = p;
+    for (int i = threadIdx.y; i < n; i += blockDim.y) {
+        float p = 0.f;
+        if (j < m)
+            for (int c = 0; c < chunks; ++c) p += partial[(int64_t)c * total + (int64_t)i * m + j];
+        message[i][threadIdx.x] = p;
+    }
     __syncthreads();
-    if (i != 0 || j >= m) return;
+    if (threadIdx.y != 0 || j >= m) return;
     float s = 0.f;
     for (int r = 0; r < n; ++r) s += message[r][threadIdx.x];
     pbar[j] = s / (float)n;
@@ -337,7 +339,8 @@ void project_force_kernel(int kind) { g_force_kernel = kind; }
 
 int32_t project_group(int32_t n_left, int32_t m) {
     if (n_left > kMaxGroup && g_force_kernel != 0 && g_force_kernel != 1) {
-        const int32_t wide = n_left < kMaxGroupTc ? n_left : kMaxGroupTc;
+        const int32_t most = project_tc_max_group(m);
+        const int32_t wide = n_left < most ? n_left : most;
         if (g_force_kernel == 2 || project_tc_applies(wide, m)) return wide;
     }
     return n_left < kMaxGroup ? n_left : kMaxGroup;
@@ -345,7 +348,7 @@ int32_t project_group(int32_t n_left, int32_t m) {
 
 ProjectPlan make_project_plan(int32_t n_group, int32_t m, int64_t d, int dtype, int sm_count) {
     ProjectPlan p{};
-    const bool tc = g_force_kernel == 2 ? n_group <= kMaxGroupTc : (g_force_kernel < 0 && project_tc_applies(n_group, m));
+    const bool tc = g_force_kernel == 2 ? n_group <= project_tc_max_group(m) : (g_force_kernel < 0 && project_tc_applies(n_group, m));
     if (tc) {
         fill_project_tc_plan(p, n_group, m, d, dtype, sm_count);
         return p;
@@ -443,7 +446,7 @@ cudaError_t launch_finish_project(const float *partial, int chunks, int32_t n, i
 
 cudaError_t launch_finish_aggregate(const float *partial, int chunks, int32_t n, int32_t m, float *pbar,
                                     cudaStream_t stream) {
-    finish_aggregate_kernel<<<(m + 31) / 32, dim3(32, n > kMaxGroup ? kMaxGroupTc : kMaxGroup), 0, stream>>>(
+    finish_aggregate_kernel<<<(m + 31) / 32, dim3(32, n > kMaxGroup ? 32 : kMaxGroup), 0, stream>>>(
         partial, chunks, n, m, pbar);
     return cudaGetLastError();
 }

@@ -31,12 +31,12 @@ namespace {
 constexpr int kTcWarps = 8;
 constexpr int kTcThreads = 32 * kTcWarps;
 constexpr int kTcVectors = 128;                 // M of the instruction = vectors per group (a CTA owns VG groups)
-constexpr int kTcMaxN = 32;                     // largest N of the instruction = machines per pass (16 or 32)
+constexpr int kTcMaxN = 64;                     // largest N of the instruction = machines per pass (16, 32 or 64)
 constexpr int kTcMinMachines = 9;               // fewer machines: the scalar kernel is used
 constexpr int kTcStageBlocks = 8;               // coordinate blocks per stage: 32 coordinates = 128 B per row
 constexpr int kTcTileStages = 8;                // stages between two drains of the accumulators
 constexpr int kTcTileBlocks = kTcStageBlocks * kTcTileStages;       // 64 blocks = 256 coordinates
-// Geometry that depends on N (machines per pass: 16 or 32), on the gradients' type and on VG (groups of
+// Geometry that depends on N (machines per pass: 16, 32 or 64; 64 with two groups only), on the gradients' type and on VG (groups of
 // 128 vectors per CTA).  bf16 gradients are exact in tf32 and need one plane, fp32 gradients a head and a
 // tail plane.  With one group two CTAs share an SM (about 113 KB of shared memory each); with two groups a
 // CTA has the SM to itself, every thread generates eight counters per stage instead of four, and the
@@ -57,6 +57,10 @@ struct TcShape {
     static constexpr int kPieces = VG * NT / 16;
     static constexpr int kDrainWarps = kPieces > 1 ? 8 : 4;
     static constexpr int kPiecesPerWarp = kPieces > 2 ? kPieces / 2 : 1;
+    // Staging of the gradients: 16-byte pieces per stage, one or two per thread of the warps on duty.
+    static constexpr int kPiecesB = NT * (BF16 ? 4 : 8);
+    static constexpr int kDutyWarps = kPiecesB / 32 < kTcWarps ? kPiecesB / 32 : kTcWarps;
+    static constexpr int kDutyPieces = kPiecesB / (32 * kDutyWarps);   // per thread on duty
     // Instruction descriptor: fp32 accumulator (1 at bit 4), tf32 A and B (2 at bits 7 and 10), both
     // K-major, N >> 3 at bit 17, M >> 4 at bit 24.
     static constexpr uint32_t kIdesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(NT >> 3) << 17) |
@@ -340,39 +344,55 @@ project_tc_kernel(const __grid_constant__ TcArgs a) {
     // Gradient staging is shared out among the warps in turn: DUTY warps serve a stage, one 16-byte piece
     // per thread, fetched one stage ahead so that the load is in flight while the previous stage is
     // generated.
-    constexpr int DUTY = NT * (BF16 ? 4 : 8) / 32;                  // warps on duty per stage (one 16-byte piece per thread)
+    constexpr int DUTY = Shape::kDutyWarps;                          // warps on duty per stage
+    constexpr int PPT = Shape::kDutyPieces;                           // 16-byte pieces per thread on duty (1 or 2)
     constexpr uint32_t ROTA = kTcWarps / DUTY;                        // stages until a warp's turn comes again
     const uint32_t duty_phase = (uint32_t)warp / DUTY;                // serves stages c with c % ROTA == duty_phase
     const uint32_t fetch_phase = (duty_phase + ROTA - 1) % ROTA;      // and fetches for them one stage earlier
-    const int duty_piece = (warp % DUTY) * 32 + lane;                 // always the same 16-byte piece of the stage
-    const int duty_i = BF16 ? duty_piece >> 2 : duty_piece >> 3;      // machine
-    const int duty_c = BF16 ? duty_piece & 3 : duty_piece & 7;        // piece of the machine's row
-    const uint32_t duty_off = 2 * kTcPlaneA + plane_offset(duty_i, BF16 ? 2 * duty_c : duty_c);
     const int64_t range_begin = tile_begin * (int64_t)(4 * kTcTileBlocks);
     const int64_t range_end = min(tile_end * (int64_t)(4 * kTcTileBlocks), a.d);
     // stages of this CTA: the first `fast_stages` lie wholly inside d and can be read 16 bytes at a time
     const uint32_t total_stages = range_end > range_begin ? (uint32_t)((range_end - range_begin + 31) >> 5) : 0u;
     const uint32_t fast_stages = a.aligned && range_end > range_begin ? (uint32_t)((range_end - range_begin) >> 5) : 0u;
-    const GT *const duty_src = G + (int64_t)duty_i * a.ldg + range_begin + (BF16 ? 8 : 4) * duty_c;
-    uint4 held = make_uint4(0, 0, 0, 0);
-    auto fetch = [&](uint32_t c) {                                    // piece of stage c, if it can be read whole
-        if (c < fast_stages && duty_i < a.n) held = __ldg(reinterpret_cast<const uint4 *>(duty_src + (int64_t)c * 32));
+    int duty_i[PPT], duty_c[PPT];                                     // machine, piece of the machine's row
+    uint32_t duty_off[PPT];
+    const GT *duty_src[PPT];
+    uint4 held[PPT];
+#pragma unroll
+    for (int r = 0; r < PPT; ++r) {
+        const int piece = ((warp % DUTY) * 32 + lane) + r * (DUTY * 32);   // always the same pieces of the stage
+        duty_i[r] = BF16 ? piece >> 2 : piece >> 3;
+        duty_c[r] = BF16 ? piece & 3 : piece & 7;
+        duty_off[r] = 2 * kTcPlaneA + plane_offset(duty_i[r], BF16 ? 2 * duty_c[r] : duty_c[r]);
+        duty_src[r] = G + (int64_t)duty_i[r] * a.ldg + range_begin + (BF16 ? 8 : 4) * duty_c[r];
+        held[r] = make_uint4(0, 0, 0, 0);
+    }
+    auto fetch = [&](uint32_t c) {                                    // pieces of stage c, if they can be read whole
+        if (c < fast_stages) {
+#pragma unroll
+            for (int r = 0; r < PPT; ++r)
+                if (duty_i[r] < a.n) held[r] = __ldg(reinterpret_cast<const uint4 *>(duty_src[r] + (int64_t)c * 32));
+        }
     };
     auto deposit = [&](uint32_t c, uint32_t sb) {                     // stage c into the buffer at sb
-        const uint32_t dst = sb + duty_off;
-        if (c < fast_stages) {
-            const uint4 h = duty_i < a.n ? held : make_uint4(0, 0, 0, 0);
-            if constexpr (BF16) {
-                st_shared_v4(dst, __uint_as_float(h.x << 16), __uint_as_float(h.x & 0xFFFF0000u),
-                             __uint_as_float(h.y << 16), __uint_as_float(h.y & 0xFFFF0000u));
-                st_shared_v4<kLbo>(dst, __uint_as_float(h.z << 16), __uint_as_float(h.z & 0xFFFF0000u),
-                                   __uint_as_float(h.w << 16), __uint_as_float(h.w & 0xFFFF0000u));
+#pragma unroll
+        for (int r = 0; r < PPT; ++r) {
+            const uint32_t dst = sb + duty_off[r];
+            if (c < fast_stages) {
+                const uint4 h = duty_i[r] < a.n ? held[r] : make_uint4(0, 0, 0, 0);
+                if constexpr (BF16) {
+                    st_shared_v4(dst, __uint_as_float(h.x << 16), __uint_as_float(h.x & 0xFFFF0000u),
+                                 __uint_as_float(h.y << 16), __uint_as_float(h.y & 0xFFFF0000u));
+                    st_shared_v4<kLbo>(dst, __uint_as_float(h.z << 16), __uint_as_float(h.z & 0xFFFF0000u),
+                                       __uint_as_float(h.w << 16), __uint_as_float(h.w & 0xFFFF0000u));
+                } else {
+                    store_split_b<kTcPlaneB>(dst, __uint_as_float(h.x), __uint_as_float(h.y), __uint_as_float(h.z), __uint_as_float(h.w));
+                }
             } else {
-                store_split_b<kTcPlaneB>(dst, __uint_as_float(h.x), __uint_as_float(h.y), __uint_as_float(h.z), __uint_as_float(h.w));
+                stage_piece_slowly<GT, kTcPlaneB>(G, a.ldg, a.d, a.n, duty_i[r],
+                                                  range_begin + (int64_t)c * 32 + (BF16 ? 8 : 4) * duty_c[r], dst);
             }
-            return;
         }
-        stage_piece_slowly<GT, kTcPlaneB>(G, a.ldg, a.d, a.n, duty_i, range_begin + (int64_t)c * 32 + (BF16 ? 8 : 4) * duty_c, dst);
     };
 
     // Products of one finished stage, issued by one lane.  `st` is the stage's index in its tile of
@@ -540,19 +560,21 @@ cudaError_t launch_wait_timeout_probe(uint64_t limit_ns, int code, uint32_t *obs
     return cudaGetLastError();
 }
 
-bool project_tc_applies(int32_t n_group, int32_t m) {
-    // enough machines for the tensor core to pay (with five or more the multiply-adds of the scalar kernel cost
-    // more issue slots than this kernel's staging and hand-over), enough vectors to fill most of the 128 rows
-    // of the last CTA row
-    return n_group >= kTcMinMachines && n_group <= kTcMaxN && m >= 96 &&
-           (m % kTcVectors == 0 || m % kTcVectors >= 64 || m >= 1024);
-}
-
 // Two groups of 128 vectors per CTA (one CTA per SM) when that leaves few rows of the last CTA row
 // empty; otherwise one group (two CTAs per SM).
 static int tc_vector_groups(int32_t m) {
     const int32_t rest = m % (2 * kTcVectors);
     return (m >= 2 * kTcVectors && (rest == 0 || rest > kTcVectors + kTcVectors / 2 || m >= 16 * kTcVectors)) ? 2 : 1;
+}
+
+int32_t project_tc_max_group(int32_t m) { return tc_vector_groups(m) == 2 ? kTcMaxN : 32; }
+
+bool project_tc_applies(int32_t n_group, int32_t m) {
+    // enough machines for the tensor core to pay (with five or more the multiply-adds of the scalar kernel cost
+    // more issue slots than this kernel's staging and hand-over), enough vectors to fill most of the 128 rows
+    // of the last CTA row
+    return n_group >= kTcMinMachines && n_group <= project_tc_max_group(m) && m >= 96 &&
+           (m % kTcVectors == 0 || m % kTcVectors >= 64 || m >= 1024);
 }
 
 template <int NT, int VG>
@@ -563,7 +585,7 @@ static size_t tc_smem_bytes(bool bf16) {
 void fill_project_tc_plan(ProjectPlan &p, int32_t n_group, int32_t m, int64_t d, int dtype, int sm_count) {
     const int vg = tc_vector_groups(m);
     p.mma = 2;
-    p.nb = n_group > 16 ? 32 : 16;     // N of the instruction
+    p.nb = n_group > 32 ? 64 : n_group > 16 ? 32 : 16;     // N of the instruction
     p.jt = 4 * vg;                     // producer thread = (lane, warp): 4 or 8 vectors x 1 block per stage
     p.uq = 1;
     p.tile_q = kTcTileBlocks;
@@ -572,7 +594,7 @@ void fill_project_tc_plan(ProjectPlan &p, int32_t n_group, int32_t m, int64_t d,
     p.grid_y = (m + vg * kTcVectors - 1) / (vg * kTcVectors);
     p.tiles = (d + 4 * (int64_t)kTcTileBlocks - 1) / (4 * (int64_t)kTcTileBlocks);
     const bool bf16 = dtype == 1;
-    if (vg == 2) p.smem = p.nb == 32 ? tc_smem_bytes<32, 2>(bf16) : tc_smem_bytes<16, 2>(bf16);
+    if (vg == 2) p.smem = p.nb == 64 ? tc_smem_bytes<64, 2>(bf16) : p.nb == 32 ? tc_smem_bytes<32, 2>(bf16) : tc_smem_bytes<16, 2>(bf16);
     else p.smem = p.nb == 32 ? tc_smem_bytes<32, 1>(bf16) : tc_smem_bytes<16, 1>(bf16);
     int64_t gx = (int64_t)sm_count * (vg == 2 ? 1 : 2) / p.grid_y;
     if (gx < 1) gx = 1;
@@ -583,7 +605,8 @@ void fill_project_tc_plan(ProjectPlan &p, int32_t n_group, int32_t m, int64_t d,
 cudaError_t launch_project_tc(const ProjectPlan &plan, const RoundKeys &keys, uint32_t t, const void *G, int dtype,
                               int32_t n, int64_t ldg, int64_t d, int32_t m, uint64_t q_base, float *partial,
                               cudaStream_t stream) {
-    if (q_base % kTcTileBlocks != 0 || n > plan.nb || (plan.nb != 16 && plan.nb != 32) || (plan.jt != 4 && plan.jt != 8))
+    if (q_base % kTcTileBlocks != 0 || n > plan.nb || (plan.nb != 16 && plan.nb != 32 && plan.nb != 64) ||
+        (plan.jt != 4 && plan.jt != 8) || (plan.nb == 64 && plan.jt != 8))
         return cudaErrorInvalidValue;
     TcArgs a{};
     a.G = G;
@@ -614,7 +637,8 @@ cudaError_t launch_project_tc(const ProjectPlan &plan, const RoundKeys &keys, ui
     using I32 = std::integral_constant<int, 32>;
     using I1 = std::integral_constant<int, 1>;
     using I2 = std::integral_constant<int, 2>;
-    if (plan.jt == 8) return plan.nb == 32 ? pick(I32{}, I2{}) : pick(I16{}, I2{});
+    using I64 = std::integral_constant<int, 64>;
+    if (plan.jt == 8) return plan.nb == 64 ? pick(I64{}, I2{}) : plan.nb == 32 ? pick(I32{}, I2{}) : pick(I16{}, I2{});
     return plan.nb == 32 ? pick(I32{}, I1{}) : pick(I16{}, I1{});
 }
 

@@ -55,14 +55,15 @@ def test_project_plans_are_consistent():
     """Launch geometry (host logic): the thread grid covers all m vectors and all tiles of d,
     the per-thread stepping divides a tile, and the shared memory fits an SM."""
     from paper_2309_13307_b200 import binding
-    for n in (1, 2, 3, 4, 8, 16, 40):
+    for n in (1, 2, 3, 4, 8, 16, 40, 70):
         for m in (1, 2, 8, 64, 511, 512, 1030, 4096, 100_000):
             for d in (1, 4097, 25_557_032, 1_000_000_000):
                 for dtype in (binding.CORE_F32, binding.CORE_BF16):
                     p = binding.core_debug_project_plan(n, m, d, dtype, 148)
                     tensor_memory = (p["tj"], p["tq"], p["tile_q"]) == (32, 8, 64)
-                    assert p["nb"] >= min(n, 16) and p["nb"] in (1, 2, 4, 8, 16, 32)
+                    assert p["nb"] >= min(n, 16) and p["nb"] in (1, 2, 4, 8, 16, 32, 64)
                     assert p["nb"] <= 16 or (tensor_memory and n > 16 and m >= 96)
+                    assert p["nb"] <= 32 or (n > 32 and p["jt"] == 8)        # 64 machines need 256 vectors per CTA
                     assert p["tj"] * p["tq"] == 256
                     assert p["tile_q"] % (p["tq"] * p["uq"]) == 0
                     assert p["grid_y"] * p["tj"] * p["jt"] >= m

@@ -87,7 +87,11 @@ def test_ragged_sizes(core_mod, d, m, n):
     (32, 256, 30_011, "f32", "scaled_normal"),   # 32 machines in one pass (N = 32 of the instruction), fp32: two-stage ring
     (32, 256, 30_011, "bf16", "student_t3"),     # the same with one gradient plane and a three-stage ring
     (50, 130, 9_001, "f32", "normal"),           # 32 + 18 machines
-    (64, 1024, 5_003, "bf16", "normal"),         # 32 + 32
+    (64, 1024, 5_003, "bf16", "normal"),         # 64 machines in one pass (N = 64, 256 vectors per CTA)
+    (50, 256, 30_011, "f32", "normal"),          # 50 machines, fp32: N = 64 with a two-stage ring
+    (33, 512, 9_001, "f32", "scaled_normal"),    # 33 machines: N = 64 with 31 empty columns
+    (64, 128, 9_001, "bf16", "normal"),          # 64 machines, 128 vectors: two passes of 32
+    (70, 256, 9_001, "bf16", "student_t3"),      # 64 + 6
     (17, 96, 70_001, "bf16", "scaled_normal"),   # 17 machines: N = 32 with 15 empty columns
     (16, 456, 30_001, "f32", "normal"),          # two groups of 128 vectors per CTA, second CTA row 200 of 256 full
     (20, 456, 30_001, "bf16", "student_t3"),     # the same with N = 32
@@ -128,6 +132,7 @@ def test_device_status_word(core_mod):
     (10, 70, "f32"), (12, 72, "bf16"),                    # warp-level tensor-core projection
     (16, 256, "bf16"), (9, 128, "f32"),                   # tcgen05 projection
     (32, 128, "f32"), (27, 256, "bf16"),                  # tcgen05 projection, 32 machines per pass
+    (64, 256, "bf16"), (40, 512, "f32"),                  # tcgen05 projection, 64 machines per pass
 ])
 def test_unit_vectors_read_the_generator_back(core_mod, n, m, dtype):
     """Machine i holds the unit vector e_k(i): its message is p_ij = xi_j[k(i)], and every other term of
