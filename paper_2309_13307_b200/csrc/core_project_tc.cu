@@ -7,12 +7,14 @@
 // head and tail (z = hi + lo, both exact in fp32) and writes the two planes to shared memory in the
 // K-major core-matrix layout the tensor core reads; in turn the warps also stage the machines' gradients
 // for the same 32 coordinates (split the same way when they are fp32; bf16 is exact in tf32).  The
-// products of stage c are issued by one lane of warp c % 8 once it has finished generating stage c + 1
-// (and before it reports that stage done, which keeps the issue order equal to the stage order): per 8
-// coordinates  tcgen05.mma  D[128 vectors x 16 machines] += A[128 x 8] * B[8 x 16]  for hi*hi, lo*hi
-// (and hi*lo for fp32 gradients).  D lives in tensor memory, double buffered, with the small products in
-// an accumulator of their own: every 8 stages (256 coordinates) four warps move both to registers with
-// tcgen05.ld and add them to fp32 running sums.  The tensor core's accumulator loses about half an ulp
+// products of stage c are issued by one elected lane of warp c % 8 once it has finished generating stage
+// c + 1 (and before it reports that stage done, which keeps the issue order equal to the stage order); the
+// descriptors are computed by the whole warp from warp-uniform values, so they stay in uniform registers.
+// Per group of 128 vectors and 8 coordinates:  tcgen05.mma  D[128 vectors x N machines] += A[128 x 8] *
+// B[8 x N]  (N = 16, 32 or 64) for hi*hi, lo*hi (and hi*lo for fp32 gradients).  D lives in tensor
+// memory, double buffered, with the small products in an accumulator of their own: every 8 stages (256
+// coordinates) the warps move both to registers with tcgen05.ld (a piece of 32 vectors x 16 machines at a
+// time) and add them to fp32 running sums.  The tensor core's accumulator loses about half an ulp
 // of the running sum per product, always in the same direction, so its chains are kept short and the
 // large and small terms apart.  Stage buffers and accumulators are handed over with mbarriers; every
 // wait is bounded, and a wait that runs out sets a device status word and lets the CTA leave through the
