@@ -40,7 +40,7 @@ WIDE_MULS_PER_GAUSSIAN = 4
 # multiply-adds and 64 for logic ops; Philox's rounds 2..9 alone take 75.2 scheduler cycles per warp and counter.
 WIDE_MUL_LANES_PER_CLK_SM = 32
 PHILOX_ONLY_CYCLES_PER_COUNTER = 75.2
-# Planning count of the survey's issue bound: 16 lane-instructions per Gaussian for the generator plus the
+# Planning count of the plain issue bound: 16 lane-instructions per Gaussian for the generator plus the
 # consumer's multiply-adds (n per pair in the projection, 1 in the reconstruction), 128 lanes per clock per SM.
 PLANNING_INSTR_PER_GAUSSIAN = 16
 ISSUE_LANES_PER_CLK_SM = 128
@@ -55,7 +55,7 @@ def alu_bounds(sm_max_mhz: float):
 
 
 def planning_bound(sm_max_mhz: float, fmas_per_pair: int) -> float:
-    """The survey's issue bound R / (c_g + c_f) in pairs per second."""
+    """The plain issue bound R / (c_g + c_f) in pairs per second."""
     return SM_COUNT * ISSUE_LANES_PER_CLK_SM * sm_max_mhz * 1e6 / (PLANNING_INSTR_PER_GAUSSIAN + fmas_per_pair)
 
 
