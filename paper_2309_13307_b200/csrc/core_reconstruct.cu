@@ -49,16 +49,21 @@ __device__ __forceinline__ void rec_step(const uint4 *entries, const QPart (&qp)
 #pragma unroll
         for (int u = 0; u < kRecUQ; ++u) w[s * kRecUQ + u] = philox_combine(jp, qp[u], keys);
     }
-    float4 z[JS * kRecUQ];
-    box_muller4xN<JS * kRecUQ>(w, z);
+    BmParts r[JS * kRecUQ];
+    box_muller_parts<JS * kRecUQ>(w, r);
+    // pbar_j xi_j with the message meeting the radius first: ((pbar S) y) sp and (pbar S) cs, four packed
+    // instructions per call instead of five, and xi_j itself (pbar = 1) bit for bit what the projection
+    // multiplies with.  Accumulator lanes: (x, z) = cosine lanes of pair a, b; (y, w) = sine lanes.
 #pragma unroll
     for (int s = 0; s < JS; ++s) {
 #pragma unroll
         for (int u = 0; u < kRecUQ; ++u) {
-            const float4 zz = z[s * kRecUQ + u];
-            const float2 lo = __ffma2_rn(make_float2(p[s], p[s]), make_float2(zz.x, zz.y), make_float2(acc[u].x, acc[u].y));
-            const float2 hi = __ffma2_rn(make_float2(p[s], p[s]), make_float2(zz.z, zz.w), make_float2(acc[u].z, acc[u].w));
-            acc[u] = make_float4(lo.x, lo.y, hi.x, hi.y);
+            const BmParts rr = r[s * kRecUQ + u];
+            const float2 ps = __fmul2_rn(make_float2(p[s], p[s]), rr.s);
+            const float2 psy = __fmul2_rn(ps, rr.y);
+            const float2 c2 = __ffma2_rn(psy, rr.sp, make_float2(acc[u].x, acc[u].z));
+            const float2 s2 = __ffma2_rn(ps, rr.cs, make_float2(acc[u].y, acc[u].w));
+            acc[u] = make_float4(c2.x, s2.x, c2.y, s2.y);
         }
     }
 }

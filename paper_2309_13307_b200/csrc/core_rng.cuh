@@ -181,31 +181,47 @@ __device__ __forceinline__ void bm_fix_near_one(uint4 w, float2 u, float2 &l) {
 }
 
 // The rest of Box-Muller given l with |l| = -log2 u of the two pairs (the sign of l is ignored:
-// the hardware path delivers log2 u < 0, the correction delivers the positive series).
-__device__ __forceinline__ float4 bm_finish(uint4 w, float2 l) {
-    float2 s;
-    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(s.x) : "f"(fabsf(l.x)));
-    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(s.y) : "f"(fabsf(l.y)));
+// the hardware path delivers log2 u < 0, the correction delivers the positive series), as its factors:
+// with S = (-1)^h sqrt(-log2 u) the pair is (r cos theta, r sin theta) = ((S y) sp, S cs).  Lanes x, y of
+// every member = pair a, pair b.  A consumer that multiplies the values by a number p of its own can let p
+// meet S first, ((p S) y) sp and (p S) cs, and save the two products that would form the values; with
+// p = 1 that is bit for bit what bm_finish returns.
+struct BmParts {
+    float2 s;     // (-1)^h sqrt(-log2 u)
+    float2 y;     // f - 1/2
+    float2 sp;    // -sqrt(2 ln 2) sin(pi y) / y
+    float2 cs;    //  sqrt(2 ln 2) cos(pi y)
+};
+
+__device__ __forceinline__ BmParts bm_parts(uint4 w, float2 l) {
+    BmParts r;
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r.s.x) : "f"(fabsf(l.x)));
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r.s.y) : "f"(fabsf(l.y)));
 
     // angles: theta = pi (h + f), h = bit 31 of the word, f = (bits 30..9 + 1/2) / 2^22 in (0, 1).
     // With y = f - 1/2:  cos theta = -(-1)^h sin(pi y),  sin theta = (-1)^h cos(pi y).
-    const float2 y = __fadd2_rn(make_float2(__uint_as_float(((w.y >> 8) & 0x007FFFFEu) | 0x3F800001u),
-                                            __uint_as_float(((w.w >> 8) & 0x007FFFFEu) | 0x3F800001u)),
-                                bm_splat(-1.5f));
-    s.x = __uint_as_float(__float_as_uint(s.x) ^ (w.y & 0x80000000u));
-    s.y = __uint_as_float(__float_as_uint(s.y) ^ (w.w & 0x80000000u));
-    const float2 y2 = __fmul2_rn(y, y);
+    r.y = __fadd2_rn(make_float2(__uint_as_float(((w.y >> 8) & 0x007FFFFEu) | 0x3F800001u),
+                                 __uint_as_float(((w.w >> 8) & 0x007FFFFEu) | 0x3F800001u)),
+                     bm_splat(-1.5f));
+    r.s.x = __uint_as_float(__float_as_uint(r.s.x) ^ (w.y & 0x80000000u));
+    r.s.y = __uint_as_float(__float_as_uint(r.s.y) ^ (w.w & 0x80000000u));
+    const float2 y2 = __fmul2_rn(r.y, r.y);
     // -sqrt(2 ln 2) sin(pi y) / y and sqrt(2 ln 2) cos(pi y)
     float2 sp = __ffma2_rn(bm_splat(-0.09091975539922714f), y2, bm_splat(0.7041443586349487f));
     sp = __ffma2_rn(sp, y2, bm_splat(-3.0024325847625732f));
     sp = __ffma2_rn(sp, y2, bm_splat(6.08450984954834f));
-    sp = __ffma2_rn(sp, y2, bm_splat(-3.6989426612854004f));
+    r.sp = __ffma2_rn(sp, y2, bm_splat(-3.6989426612854004f));
     float2 cp = __ffma2_rn(bm_splat(0.2591251730918884f), y2, bm_splat(-1.568420648574829f));
     cp = __ffma2_rn(cp, y2, bm_splat(4.778461456298828f));
     cp = __ffma2_rn(cp, y2, bm_splat(-5.810277938842773f));
-    const float2 cs = __ffma2_rn(cp, y2, bm_splat(1.1774100065231323f));
-    const float2 zs = __fmul2_rn(s, cs);                       // r sin theta
-    const float2 zc = __fmul2_rn(__fmul2_rn(s, y), sp);        // r cos theta
+    r.cs = __ffma2_rn(cp, y2, bm_splat(1.1774100065231323f));
+    return r;
+}
+
+__device__ __forceinline__ float4 bm_finish(uint4 w, float2 l) {
+    const BmParts r = bm_parts(w, l);
+    const float2 zs = __fmul2_rn(r.s, r.cs);                       // r sin theta
+    const float2 zc = __fmul2_rn(__fmul2_rn(r.s, r.y), r.sp);      // r cos theta
     return make_float4(zc.x, zs.x, zc.y, zs.y);
 }
 
@@ -226,6 +242,24 @@ __device__ __forceinline__ void box_muller4xN(const uint4 (&w)[N], float4 (&z)[N
     }
 #pragma unroll
     for (int c = 0; c < N; ++c) z[c] = bm_finish(w[c], l[c]);
+}
+
+// The factors of N calls (same near-one handling as box_muller4xN).
+template <int N>
+__device__ __forceinline__ void box_muller_parts(const uint4 (&w)[N], BmParts (&r)[N]) {
+    float2 u[N], l[N];
+    uint32_t top = 0u;
+#pragma unroll
+    for (int c = 0; c < N; ++c) {
+        l[c] = bm_log2(w[c], u[c]);
+        top = __vimax3_u32(top, w[c].x, w[c].z);
+    }
+    if (top >= kNearOneWord) {
+#pragma unroll
+        for (int c = 0; c < N; ++c) bm_fix_near_one(w[c], u[c], l[c]);
+    }
+#pragma unroll
+    for (int c = 0; c < N; ++c) r[c] = bm_parts(w[c], l[c]);
 }
 
 __device__ __forceinline__ float4 box_muller4(uint4 w) {
