@@ -72,6 +72,10 @@ project_kernel(const __grid_constant__ ProjectArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float4 *stage0 = reinterpret_cast<float4 *>(smem_raw);
     float4 *stage1 = stage0 + NB * TILE_Q;
+    // the block-dependent half of Philox for every block of a tile, tabulated once per CTA and tile
+    // ({hi_b, lo_b, w3, -}; double buffered like the gradient tile) instead of once per thread and step
+    uint4 *qtab0 = reinterpret_cast<uint4 *>(stage1 + NB * TILE_Q);
+    uint4 *qtab1 = qtab0 + TILE_Q;
 
     const int tid = threadIdx.x;
     const int tj = a.tj;
@@ -173,8 +177,17 @@ project_kernel(const __grid_constant__ ProjectArgs a) {
         }
     };
 
+    auto fill_qtab = [&](int64_t tile, uint4 *tab) {
+        const uint32_t first = (uint32_t)(a.q_base + (uint64_t)tile * TILE_Q);
+        for (int e = tid; e < TILE_Q; e += kThreads) {
+            const QPart qp = philox_qpart(first + (uint32_t)e, a.t, a.keys);
+            tab[e] = make_uint4(qp.hi_b, qp.lo_b, qp.w3, 0u);
+        }
+    };
+
     if (tile_begin < tile_end) {
         begin_stage(tile_begin, stage0);
+        fill_qtab(tile_begin, qtab0);
         finish_stage(tile_begin, stage0);
     }
     cp_async_wait_all();
@@ -188,11 +201,14 @@ project_kernel(const __grid_constant__ ProjectArgs a) {
     for (int64_t tile = tile_begin; tile < tile_end; ++tile) {
         float4 *cur = ((tile - tile_begin) & 1) ? stage1 : stage0;
         float4 *nxt = ((tile - tile_begin) & 1) ? stage0 : stage1;
+        const uint4 *qtab = ((tile - tile_begin) & 1) ? qtab1 : qtab0;
         const bool more = tile + 1 < tile_end;
-        if (more) begin_stage(tile + 1, nxt);
+        if (more) {
+            begin_stage(tile + 1, nxt);
+            fill_qtab(tile + 1, ((tile - tile_begin) & 1) ? qtab0 : qtab1);
+        }
 
         const uint64_t q0 = a.q_base + (uint64_t)tile * TILE_Q;   // multiple of TILE_Q: no carry inside
-        const uint32_t q0_lo = (uint32_t)q0;
         const uint32_t q_hi = (uint32_t)(q0 >> 32);
         if (!have_jp || q_hi != jp_q_hi) {
 #pragma unroll
@@ -211,7 +227,11 @@ project_kernel(const __grid_constant__ ProjectArgs a) {
             uint4 w[UQ * JT];
 #pragma unroll
             for (int u = 0; u < UQ; ++u) {
-                const QPart qp = philox_qpart(q0_lo + (uint32_t)(qq + u), a.t, a.keys);
+                const uint4 e = qtab[qq + u];
+                QPart qp;
+                qp.hi_b = e.x;
+                qp.lo_b = e.y;
+                qp.w3 = e.z;
 #pragma unroll
                 for (int v = 0; v < JT; ++v) w[u * JT + v] = philox_combine(jp[v], qp, a.keys);
             }
@@ -388,7 +408,8 @@ ProjectPlan make_project_plan(int32_t n_group, int32_t m, int64_t d, int dtype, 
     p.tiles = (d + 4 * (int64_t)p.tile_q - 1) / (4 * (int64_t)p.tile_q);
     const size_t stage = (size_t)p.nb * p.tile_q * 16;
     const size_t red = (size_t)kThreads * p.nb * p.jt * 4;
-    p.smem = 2 * stage > red ? 2 * stage : red;
+    const size_t tiles_and_tables = 2 * stage + 2 * (size_t)p.tile_q * 16;   // two gradient tiles + two Philox block tables
+    p.smem = tiles_and_tables > red ? tiles_and_tables : red;
     int ctas_per_sm = (int)((size_t)(200 * 1024) / p.smem);
     if (ctas_per_sm > 2) ctas_per_sm = 2;
     if (ctas_per_sm < 1) ctas_per_sm = 1;
